@@ -1,0 +1,182 @@
+/*
+ * rksc.h - C ABI of the B200 (sm_100a) ASKS hot path: the similarity gate and
+ * multi-branch decode attention over a paged bf16 KV pool in which every branch
+ * mapped onto a shared prefix reads that prefix's pages once.
+ *
+ * Conventions
+ *   - Every call returns an int32_t status: RKSC_OK (0) or a negative RKSC_ERR_*.
+ *     Nothing throws, prints or exits.  rksc_strerror() names a status.
+ *   - "dev" pointers are device memory owned by the caller; "host" pointers are
+ *     host memory owned by the caller.  The library never frees caller memory.
+ *     It owns only rksc_plan objects and tables filled by rksc_tables_from_gate
+ *     (released with rksc_plan_destroy / rksc_tables_free).
+ *   - Device work is enqueued on the caller's stream (a cudaStream_t passed as
+ *     void*, NULL = default stream) and is asynchronous.  The compute calls do not
+ *     synchronise the host.
+ *   - bf16 tensors are passed as const void* (2 bytes per element).
+ *   - The device must be compute capability 10.x; other devices give
+ *     RKSC_ERR_UNSUPPORTED.
+ */
+#ifndef RKSC_H_
+#define RKSC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RKSC_OK                   0
+#define RKSC_ERR_INVALID_ARG     (-1)  /* NULL pointer, non-positive size, misaligned buffer       */
+#define RKSC_ERR_UNSUPPORTED     (-2)  /* head_dim not 64/128, block_size not 16, device not sm_100 */
+#define RKSC_ERR_BAD_TABLE       (-3)  /* page id out of range, token count inconsistent with pages */
+#define RKSC_ERR_WORKSPACE       (-4)  /* workspace too small or misaligned                         */
+#define RKSC_ERR_CUDA            (-5)  /* a CUDA runtime/driver call failed (or no device present)  */
+#define RKSC_ERR_DEVICE_TIMEOUT  (-6)  /* value a kernel writes to device_status when a wait ran out */
+#define RKSC_ERR_NOMEM           (-7)  /* host allocation failed                                    */
+
+#define RKSC_BLOCK_SIZE 16
+
+#if defined(__GNUC__)
+#define RKSC_API __attribute__((visibility("default")))
+#else
+#define RKSC_API
+#endif
+
+RKSC_API const char* rksc_strerror(int32_t status);
+
+/* ------------------------------------------------------------------------------------------
+ * ASKS similarity gate  (paper Eq. 2 and Algorithm 2)
+ *
+ *   w_l     = exp(alpha*l/L) / sum_l' exp(alpha*l'/L),  l = 1..L
+ *   sigma_b = sum_l w_l * <h_b^l, h_r^l> / (|h_b^l| |h_r^l|),   r = cand_prefix[b]
+ *   branch_to_prefix[b] = r if sigma_b >= tau else -1           (">=": Alg. 2 line 6)
+ *
+ * h_branch  dev [B][L][D] fp32, one vector per (branch, layer)
+ * h_root    dev [P][L][D] fp32, raw or already unit-norm (the norm is always divided out)
+ * cand_prefix dev [B] int32 in [0,P): the root each branch is compared with
+ * branch_to_prefix dev [B] int32 out; sigma dev [B] fp32 out, may be NULL
+ * A zero-norm vector contributes 0 for its layer; NaN inputs give -1.  An out-of-range
+ * candidate gives -1 and sigma = NaN.  Arithmetic is fp32 (tree reductions): the map is
+ * exact whenever |sigma - tau| is above ~1e-5.
+ * One kernel launch on `stream`; no workspace.  D and L are arbitrary positive sizes
+ * (16-byte loads are used when D % 4 == 0 and both bases are 16-byte aligned).
+ * ------------------------------------------------------------------------------------------ */
+RKSC_API int32_t rksc_asks_gate(const float* h_branch, const float* h_root, const int32_t* cand_prefix,
+                       int32_t B, int32_t P, int32_t L, int32_t D,
+                       float alpha, float tau,
+                       int32_t* branch_to_prefix, float* sigma, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * KV pool layout and block tables
+ *
+ * Pool: K and V are separate dev tensors [num_pool_blocks][num_kv_heads][16][head_dim] bf16,
+ * 16-byte aligned.  Query head h reads KV head h / (num_q_heads / num_kv_heads).
+ *
+ * Tables (segment form): segment s owns pages seg_blocks[seg_block_off[s] .. seg_block_off[s+1])
+ * and seg_num_tokens[s] tokens; every page but the last is full, the last holds at least one
+ * token (a segment may also be empty: no pages, 0 tokens).  Branch b attends to the segments
+ * br_segs[br_seg_off[b] .. br_seg_off[b+1]) in that (root-to-leaf) order; a segment listed by
+ * several branches is a shared prefix.  This is what replaces the B physical copies of the
+ * prefix cache that the paper's Algorithm 1 (line 3) makes.
+ * The "logical block" j of a branch is the j-th page of that concatenation.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    int32_t num_q_heads;
+    int32_t num_kv_heads;
+    int32_t head_dim;         /* 64 or 128 */
+    int32_t block_size;       /* 16 */
+    float   sm_scale;         /* <= 0 selects 1/sqrt(head_dim) */
+    int32_t num_pool_blocks;
+} rksc_layout;
+
+typedef struct {
+    int32_t num_branches;
+    int32_t num_segments;
+    const int32_t* seg_block_off;   /* host [S+1] */
+    const int32_t* seg_blocks;      /* host, physical page ids */
+    const int32_t* seg_num_tokens;  /* host [S]   */
+    const int32_t* br_seg_off;      /* host [B+1] */
+    const int32_t* br_segs;         /* host       */
+} rksc_tables;
+
+/* Tables from a gate map for the two-level case (P shared prefixes; per branch a private
+ * prefix copy and a suffix).  All arguments are host pointers; *_off are CSR offsets into the
+ * page-id arrays, *_ntok the token counts.  Branch b uses shared prefix branch_to_prefix[b]
+ * when that is >= 0 and otherwise its private prefix list (the paper's "independent
+ * recomputation" for branches below tau, Section 2.2), followed by its suffix.
+ * Segment numbering: shared prefixes by ascending id (only those with a sharer), private
+ * prefixes of the non-sharing branches by ascending branch, then all suffixes by ascending
+ * branch.  `out` is filled with arrays the library allocates; release with rksc_tables_free.
+ * Errors: RKSC_ERR_INVALID_ARG (NULL, map entry >= P), RKSC_ERR_NOMEM. */
+RKSC_API int32_t rksc_tables_from_gate(int32_t B, int32_t P, const int32_t* branch_to_prefix,
+                              const int32_t* shared_off, const int32_t* shared_pages, const int32_t* shared_ntok,
+                              const int32_t* priv_off,   const int32_t* priv_pages,   const int32_t* priv_ntok,
+                              const int32_t* sfx_off,    const int32_t* sfx_pages,    const int32_t* sfx_ntok,
+                              rksc_tables* out);
+RKSC_API void rksc_tables_free(rksc_tables* t);
+
+/* ------------------------------------------------------------------------------------------
+ * Plan: validated tables turned into device work lists.
+ *
+ * rksc_plan_create checks the tables (RKSC_ERR_BAD_TABLE), groups each segment with the
+ * ascending list of branches that share it, cuts segments into KV chunks sized for the
+ * device's SM count, lays out the partial-result workspace and the block-mass output, and
+ * uploads its lists to the current device (synchronously; it may allocate device memory).
+ * Without a CUDA device the plan is host-only: it can be queried but not run.
+ * A plan is immutable and may be used from several streams at once with distinct
+ * workspaces.  It does not keep pointers into `tables`.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct rksc_plan rksc_plan;
+
+typedef struct {
+    size_t  workspace_bytes;     /* required size of the attention workspace              */
+    int64_t mass_elems;          /* floats in block_mass: num_q_heads * sum_b nblk_b      */
+    const int64_t* mass_off;     /* host [B+1], owned by the plan: sum of nblk over b' < b */
+    int32_t num_work_items;      /* CTAs of the segment-attention launch                  */
+    int32_t num_partial_rows;    /* (row, chunk) partial results merged at the end        */
+    int64_t unique_kv_tokens;    /* valid tokens of the distinct segments referenced       */
+    int64_t duplicated_kv_tokens;/* sum over branches of the tokens they attend to        */
+    int32_t on_device;           /* 1 when the lists were uploaded                        */
+} rksc_plan_info;
+
+RKSC_API int32_t rksc_plan_create(const rksc_layout* layout, const rksc_tables* tables, rksc_plan** out);
+RKSC_API int32_t rksc_plan_query(const rksc_plan* plan, rksc_plan_info* info);
+/* Work item i as 10 int32: segment, kv_head, first page (index within the segment), pages,
+ * tokens, first sharer (index within the segment's sharer list), sharers, first partial row,
+ * kernel class (0 = warp MMA), reserved.  For tests and tools. */
+RKSC_API int32_t rksc_plan_get_item(const rksc_plan* plan, int32_t i, int32_t* out10);
+RKSC_API void    rksc_plan_destroy(rksc_plan* plan);
+
+/* ------------------------------------------------------------------------------------------
+ * Branch-decode attention  (the attention inside the paper's batched decode on the shared
+ * cache: Algorithm 1 line 4, Section 2.2 "KV broadcast and batched decode")
+ *
+ *   out[b][h][:]       = softmax_j(scale * q[b][h] . k_j) V     over all tokens j of branch b
+ *   block_mass[b][h][j] = sum of those softmax probabilities over the tokens of logical block j
+ *
+ * q          dev [B][Hq][d] bf16 (one decode query per branch and head), 16-byte aligned
+ * k_pool, v_pool  dev bf16 pools (see above)
+ * out        dev [B][Hq][d] fp32
+ * block_mass dev fp32 or NULL; entry (b,h,j) at mass_off[b]*Hq + h*nblk_b + j; sums to 1 over
+ *            j for every (b,h) with at least one token.  This is the per-block attention score
+ *            an attention-weighted eviction policy (the paper's RSBCM, Algorithm 4) consumes.
+ * workspace  dev, >= workspace_bytes, 256-byte aligned; contents need not be initialised
+ * device_status dev int32 or NULL.  Kernels only ever write a nonzero RKSC_ERR_* there (when a
+ *            bounded wait inside a kernel ran out); the caller zeroes it beforehand and reads
+ *            it after synchronising.
+ * Each prefix page shared by n branches is fetched from HBM once per KV head and serves all
+ * n * (Hq/Hkv) stacked query rows.  A branch without tokens gets out = 0.
+ * Launches: one segment-attention kernel + one merge kernel on `stream`.
+ * ------------------------------------------------------------------------------------------ */
+RKSC_API int32_t rksc_branch_decode_attention(const rksc_plan* plan, const void* q,
+                                     const void* k_pool, const void* v_pool,
+                                     float* out, float* block_mass,
+                                     void* workspace, size_t workspace_bytes,
+                                     int32_t* device_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RKSC_H_ */

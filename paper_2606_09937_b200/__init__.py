@@ -1,0 +1,23 @@
+"""B200 (sm_100a) ASKS hot path: similarity gate + shared-prefix branch-decode attention.
+
+The work is done by hand-written CUDA kernels behind a C ABI (``include/rksc.h``,
+built into ``librksc.so`` in this directory).  This package is a thin ctypes
+binding with the same entry-point names; torch is used for device memory and
+streams only.  There is no CPU or eager fallback: if the library cannot be
+loaded, importing the binding's functions raises.
+"""
+from .binding import (  # noqa: F401
+    RkscError,
+    Layout,
+    Tables,
+    Plan,
+    lib,
+    lib_path,
+    rksc_strerror,
+    rksc_asks_gate,
+    rksc_tables_from_gate,
+    rksc_plan_create,
+    rksc_branch_decode_attention,
+    split_block_mass,
+    EXPORTED_SYMBOLS,
+)

@@ -1,0 +1,288 @@
+"""ctypes binding of librksc.so: argument marshalling only.
+
+Every function mirrors the C entry point of the same name (see include/rksc.h).
+Tensors are torch CUDA tensors whose data pointers are handed to the library;
+work is enqueued on torch's current stream unless a stream is given.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG_DIR, "librksc.so")
+_lib = None
+
+EXPORTED_SYMBOLS = (
+    "rksc_strerror",
+    "rksc_asks_gate",
+    "rksc_tables_from_gate",
+    "rksc_tables_free",
+    "rksc_plan_create",
+    "rksc_plan_query",
+    "rksc_plan_get_item",
+    "rksc_plan_destroy",
+    "rksc_branch_decode_attention",
+)
+
+
+class RkscError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: {rksc_strerror(status)} (status {status})")
+
+
+class _CLayout(C.Structure):
+    _fields_ = [("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("block_size", C.c_int32), ("sm_scale", C.c_float), ("num_pool_blocks", C.c_int32)]
+
+
+class _CTables(C.Structure):
+    _fields_ = [("num_branches", C.c_int32), ("num_segments", C.c_int32),
+                ("seg_block_off", C.POINTER(C.c_int32)), ("seg_blocks", C.POINTER(C.c_int32)),
+                ("seg_num_tokens", C.POINTER(C.c_int32)), ("br_seg_off", C.POINTER(C.c_int32)),
+                ("br_segs", C.POINTER(C.c_int32))]
+
+
+class _CPlanInfo(C.Structure):
+    _fields_ = [("workspace_bytes", C.c_size_t), ("mass_elems", C.c_int64),
+                ("mass_off", C.POINTER(C.c_int64)), ("num_work_items", C.c_int32),
+                ("num_partial_rows", C.c_int32), ("unique_kv_tokens", C.c_int64),
+                ("duplicated_kv_tokens", C.c_int64), ("on_device", C.c_int32)]
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> C.CDLL:
+    """The loaded library.  Raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2606_09937_b200.build` "
+            "(needs nvcc).  This package has no CPU or eager fallback.")
+    L = C.CDLL(_LIB_PATH)
+    i32p = C.POINTER(C.c_int32)
+    L.rksc_strerror.restype = C.c_char_p
+    L.rksc_strerror.argtypes = [C.c_int32]
+    L.rksc_asks_gate.restype = C.c_int32
+    L.rksc_asks_gate.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                 C.c_int32, C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.rksc_tables_from_gate.restype = C.c_int32
+    L.rksc_tables_from_gate.argtypes = [C.c_int32, C.c_int32, i32p] + [i32p] * 9 + [C.POINTER(_CTables)]
+    L.rksc_tables_free.restype = None
+    L.rksc_tables_free.argtypes = [C.POINTER(_CTables)]
+    L.rksc_plan_create.restype = C.c_int32
+    L.rksc_plan_create.argtypes = [C.POINTER(_CLayout), C.POINTER(_CTables), C.POINTER(C.c_void_p)]
+    L.rksc_plan_query.restype = C.c_int32
+    L.rksc_plan_query.argtypes = [C.c_void_p, C.POINTER(_CPlanInfo)]
+    L.rksc_plan_get_item.restype = C.c_int32
+    L.rksc_plan_get_item.argtypes = [C.c_void_p, C.c_int32, i32p]
+    L.rksc_plan_destroy.restype = None
+    L.rksc_plan_destroy.argtypes = [C.c_void_p]
+    L.rksc_branch_decode_attention.restype = C.c_int32
+    L.rksc_branch_decode_attention.argtypes = [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p, C.c_void_p]
+    _lib = L
+    return L
+
+
+def rksc_strerror(status: int) -> str:
+    return lib().rksc_strerror(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise RkscError(status, where)
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(C.POINTER(C.c_int32))
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+class Layout:
+    """Mirror of rksc_layout."""
+
+    def __init__(self, num_q_heads, num_kv_heads, head_dim, num_pool_blocks, sm_scale=0.0, block_size=16):
+        self.c = _CLayout(int(num_q_heads), int(num_kv_heads), int(head_dim), int(block_size),
+                          float(sm_scale), int(num_pool_blocks))
+
+    @classmethod
+    def of(cls, layout) -> "Layout":
+        """From any object with the same attribute names (e.g. a workload's layout)."""
+        return cls(layout.num_q_heads, layout.num_kv_heads, layout.head_dim, layout.num_pool_blocks,
+                   getattr(layout, "sm_scale", 0.0), getattr(layout, "block_size", 16))
+
+
+class Tables:
+    """Mirror of rksc_tables over host arrays (numpy int32, kept alive here)."""
+
+    def __init__(self, seg_block_off, seg_blocks, seg_num_tokens, br_seg_off, br_segs, _owned=None):
+        self.seg_block_off = _i32(seg_block_off)
+        self.seg_blocks = _i32(seg_blocks)
+        self.seg_num_tokens = _i32(seg_num_tokens)
+        self.br_seg_off = _i32(br_seg_off)
+        self.br_segs = _i32(br_segs)
+        self.c = _CTables(len(self.br_seg_off) - 1, len(self.seg_num_tokens),
+                          _p(self.seg_block_off), _p(self.seg_blocks), _p(self.seg_num_tokens),
+                          _p(self.br_seg_off), _p(self.br_segs))
+
+    @classmethod
+    def of(cls, t) -> "Tables":
+        if isinstance(t, cls):
+            return t
+        if isinstance(t, dict):
+            return cls(t["seg_block_off"], t["seg_blocks"], t["seg_num_tokens"], t["br_seg_off"], t["br_segs"])
+        return cls(t.seg_block_off, t.seg_blocks, t.seg_num_tokens, t.br_seg_off, t.br_segs)
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k in
+                ("seg_block_off", "seg_blocks", "seg_num_tokens", "br_seg_off", "br_segs")}
+
+
+def rksc_tables_from_gate(branch_to_prefix, num_prefixes,
+                          shared_off, shared_pages, shared_ntok,
+                          priv_off, priv_pages, priv_ntok,
+                          sfx_off, sfx_pages, sfx_ntok) -> Tables:
+    """Host call: segment tables from a gate map (arrays are copied out of the library's result)."""
+    arrs = [_i32(a) for a in (branch_to_prefix, shared_off, shared_pages, shared_ntok,
+                              priv_off, priv_pages, priv_ntok, sfx_off, sfx_pages, sfx_ntok)]
+    out = _CTables()
+    st = lib().rksc_tables_from_gate(len(arrs[0]), int(num_prefixes), *[_p(a) for a in arrs], C.byref(out))
+    _check(st, "rksc_tables_from_gate")
+    try:
+        S, B = out.num_segments, out.num_branches
+        cp = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(max(n, 1),))[:n].copy()
+        seg_block_off = cp(out.seg_block_off, S + 1)
+        br_seg_off = cp(out.br_seg_off, B + 1)
+        t = Tables(seg_block_off, cp(out.seg_blocks, int(seg_block_off[-1])), cp(out.seg_num_tokens, S),
+                   br_seg_off, cp(out.br_segs, int(br_seg_off[-1])))
+    finally:
+        lib().rksc_tables_free(C.byref(out))
+    return t
+
+
+class Plan:
+    """Owner of an rksc_plan (destroyed with the object)."""
+
+    def __init__(self, handle: int, layout: Layout, tables: Tables):
+        self._h = C.c_void_p(handle)
+        self.layout = layout
+        self.tables = tables
+        info = _CPlanInfo()
+        _check(lib().rksc_plan_query(self._h, C.byref(info)), "rksc_plan_query")
+        B = tables.c.num_branches
+        self.workspace_bytes = int(info.workspace_bytes)
+        self.mass_elems = int(info.mass_elems)
+        self.mass_off = np.ctypeslib.as_array(info.mass_off, shape=(B + 1,)).copy()
+        self.num_work_items = int(info.num_work_items)
+        self.num_partial_rows = int(info.num_partial_rows)
+        self.unique_kv_tokens = int(info.unique_kv_tokens)
+        self.duplicated_kv_tokens = int(info.duplicated_kv_tokens)
+        self.on_device = bool(info.on_device)
+        self.num_branches = B
+
+    def item(self, i: int) -> np.ndarray:
+        out = np.zeros(10, dtype=np.int32)
+        _check(lib().rksc_plan_get_item(self._h, int(i), _p(out)), "rksc_plan_get_item")
+        return out
+
+    def items(self) -> np.ndarray:
+        return np.stack([self.item(i) for i in range(self.num_work_items)]) if self.num_work_items else \
+            np.zeros((0, 10), np.int32)
+
+    def close(self):
+        if self._h:
+            lib().rksc_plan_destroy(self._h)
+            self._h = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def rksc_plan_create(layout, tables) -> Plan:
+    lay = layout if isinstance(layout, Layout) else Layout.of(layout)
+    tab = Tables.of(tables)
+    h = C.c_void_p()
+    _check(lib().rksc_plan_create(C.byref(lay.c), C.byref(tab.c), C.byref(h)), "rksc_plan_create")
+    return Plan(h.value, lay, tab)
+
+
+def rksc_asks_gate(h_branch, h_root, cand_prefix, alpha: float, tau: float,
+                   branch_to_prefix=None, sigma=None, stream=None):
+    """Launches the gate kernel.  Returns (branch_to_prefix int32 [B], sigma fp32 [B]) on the device."""
+    import torch
+    assert h_branch.is_cuda and h_root.is_cuda and cand_prefix.is_cuda
+    assert h_branch.dtype == torch.float32 and h_root.dtype == torch.float32 and cand_prefix.dtype == torch.int32
+    assert h_branch.is_contiguous() and h_root.is_contiguous() and cand_prefix.is_contiguous()
+    B, L, D = h_branch.shape
+    P = h_root.shape[0]
+    assert h_root.shape[1:] == (L, D) and cand_prefix.shape == (B,)
+    if branch_to_prefix is None:
+        branch_to_prefix = torch.empty(B, dtype=torch.int32, device=h_branch.device)
+    if sigma is None:
+        sigma = torch.empty(B, dtype=torch.float32, device=h_branch.device)
+    st = lib().rksc_asks_gate(h_branch.data_ptr(), h_root.data_ptr(), cand_prefix.data_ptr(), B, P, L, D,
+                              float(alpha), float(tau), branch_to_prefix.data_ptr(), sigma.data_ptr(),
+                              _stream_ptr(stream))
+    _check(st, "rksc_asks_gate")
+    return branch_to_prefix, sigma
+
+
+def rksc_branch_decode_attention(plan: Plan, q, k_pool, v_pool, out=None, block_mass=None,
+                                 workspace=None, device_status=None, stream=None, want_mass=True):
+    """Launches the attention.  Returns (out fp32 [B][Hq][d], block_mass fp32 flat or None, device_status)."""
+    import torch
+    lay = plan.layout.c
+    B = plan.num_branches
+    assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+    assert tuple(q.shape) == (B, lay.num_q_heads, lay.head_dim)
+    for pool in (k_pool, v_pool):
+        assert pool.is_cuda and pool.dtype == torch.bfloat16 and pool.is_contiguous()
+        assert tuple(pool.shape) == (lay.num_pool_blocks, lay.num_kv_heads, 16, lay.head_dim)
+    dev = q.device
+    if out is None:
+        out = torch.empty((B, lay.num_q_heads, lay.head_dim), dtype=torch.float32, device=dev)
+    if block_mass is None and want_mass:
+        block_mass = torch.empty(max(plan.mass_elems, 1), dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device=dev)
+    if device_status is None:
+        device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = lib().rksc_branch_decode_attention(
+        plan._h, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), out.data_ptr(),
+        block_mass.data_ptr() if block_mass is not None else None,
+        workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+        device_status.data_ptr(), _stream_ptr(stream))
+    _check(st, "rksc_branch_decode_attention")
+    return out, block_mass, device_status
+
+
+def split_block_mass(plan: Plan, block_mass) -> list:
+    """The flat block_mass buffer as one [Hq][nblk_b] host array per branch."""
+    flat = block_mass.detach().cpu().numpy() if hasattr(block_mass, "detach") else np.asarray(block_mass)
+    Hq = plan.layout.c.num_q_heads
+    res = []
+    for b in range(plan.num_branches):
+        lo, hi = int(plan.mass_off[b]) * Hq, int(plan.mass_off[b + 1]) * Hq
+        res.append(flat[lo:hi].reshape(Hq, -1) if hi > lo else np.zeros((Hq, 0), np.float32))
+    return res

@@ -1,0 +1,298 @@
+// C ABI entry points: argument checks, plan upload, tensor maps, launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+#include "kernels.h"
+
+namespace {
+
+using namespace rksc;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+std::mutex g_mu;
+EncodeTiledFn g_encode = nullptr;
+constexpr int kMaxDevices = 64;
+int g_dev_state[kMaxDevices];   // 0 unknown, 1 ready (sm_100 family, kernels configured), -1 unsupported, -2 cuda error
+
+// Current device checked once: compute capability 10.x and kernel attributes set.
+int32_t ensure_device(int* dev_out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    if (dev_out) *dev_out = dev;
+    if (dev < 0 || dev >= kMaxDevices) return RKSC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (g_dev_state[dev] == 0) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+            cudaGetLastError();
+            g_dev_state[dev] = -2;
+        } else if (major != 10) {
+            g_dev_state[dev] = -1;
+        } else if (configure_attention_kernels() != cudaSuccess) {
+            cudaGetLastError();
+            g_dev_state[dev] = -2;
+        } else {
+            g_dev_state[dev] = 1;
+        }
+    }
+    if (g_dev_state[dev] == 1) return RKSC_OK;
+    return g_dev_state[dev] == -1 ? RKSC_ERR_UNSUPPORTED : RKSC_ERR_CUDA;
+}
+
+int32_t get_encode(EncodeTiledFn* fn) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_encode) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || !p) {
+            cudaGetLastError();
+            return RKSC_ERR_CUDA;
+        }
+        g_encode = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    *fn = g_encode;
+    return RKSC_OK;
+}
+
+// The pool viewed as a 2-D bf16 tensor [num_pool_blocks * Hkv * 16 rows][head_dim], fetched in
+// boxes of 16 rows x 64 columns (128 bytes) with the 128-byte swizzle.
+int32_t make_pool_map(const rksc_layout& L, const void* base, CUtensorMap* tm) {
+    EncodeTiledFn enc;
+    int32_t st = get_encode(&enc);
+    if (st != RKSC_OK) return st;
+    const cuuint64_t gdim[2] = {(cuuint64_t)L.head_dim, (cuuint64_t)L.num_pool_blocks * L.num_kv_heads * kBlock};
+    const cuuint64_t gstride[1] = {(cuuint64_t)L.head_dim * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kBlock};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? RKSC_OK : RKSC_ERR_CUDA;
+}
+
+template <typename T>
+size_t bytes_of(const std::vector<T>& v) {
+    return (v.size() * sizeof(T) + 255) / 256 * 256;
+}
+
+int32_t upload_plan(rksc_plan* p) {
+    HostPlan& H = p->host;
+    const size_t sizes[7] = {bytes_of(H.items),     bytes_of(H.seg_blocks), bytes_of(H.sharers), bytes_of(H.merge_off),
+                             bytes_of(H.merge_rows), bytes_of(H.mass_off),   bytes_of(H.br_nblk)};
+    size_t total = 0;
+    for (size_t s : sizes) total += s;
+    if (total == 0) total = 256;
+    std::vector<uint8_t> stage;
+    try {
+        stage.assign(total, 0);
+    } catch (const std::bad_alloc&) {
+        return RKSC_ERR_NOMEM;
+    }
+    const void* srcs[7] = {H.items.data(),      H.seg_blocks.data(), H.sharers.data(), H.merge_off.data(),
+                           H.merge_rows.data(), H.mass_off.data(),   H.br_nblk.data()};
+    const size_t raw[7] = {H.items.size() * sizeof(WorkItem),   H.seg_blocks.size() * 4, H.sharers.size() * sizeof(Sharer),
+                           H.merge_off.size() * 4,              H.merge_rows.size() * 4, H.mass_off.size() * 8,
+                           H.br_nblk.size() * 4};
+    size_t offs[7], off = 0;
+    for (int i = 0; i < 7; ++i) {
+        offs[i] = off;
+        if (raw[i]) std::memcpy(stage.data() + off, srcs[i], raw[i]);
+        off += sizes[i];
+    }
+    void* d = nullptr;
+    if (cudaMalloc(&d, total) != cudaSuccess) {
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    if (cudaMemcpy(d, stage.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(d);
+        return RKSC_ERR_CUDA;
+    }
+    uint8_t* base = static_cast<uint8_t*>(d);
+    p->dev_arena = d;
+    p->dev.items = reinterpret_cast<const WorkItem*>(base + offs[0]);
+    p->dev.seg_blocks = reinterpret_cast<const int32_t*>(base + offs[1]);
+    p->dev.sharers = reinterpret_cast<const Sharer*>(base + offs[2]);
+    p->dev.merge_off = reinterpret_cast<const int32_t*>(base + offs[3]);
+    p->dev.merge_rows = reinterpret_cast<const int32_t*>(base + offs[4]);
+    p->dev.mass_off = reinterpret_cast<const int64_t*>(base + offs[5]);
+    p->dev.br_nblk = reinterpret_cast<const int32_t*>(base + offs[6]);
+    p->on_device = true;
+    return RKSC_OK;
+}
+
+}  // namespace
+
+extern "C" RKSC_API const char* rksc_strerror(int32_t status) {
+    switch (status) {
+        case RKSC_OK: return "ok";
+        case RKSC_ERR_INVALID_ARG: return "invalid argument";
+        case RKSC_ERR_UNSUPPORTED: return "unsupported configuration or device";
+        case RKSC_ERR_BAD_TABLE: return "inconsistent block table";
+        case RKSC_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case RKSC_ERR_CUDA: return "CUDA call failed or no device";
+        case RKSC_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        case RKSC_ERR_NOMEM: return "out of host memory";
+        default: return "unknown status";
+    }
+}
+
+extern "C" RKSC_API int32_t rksc_asks_gate(const float* h_branch, const float* h_root, const int32_t* cand_prefix,
+                                  int32_t B, int32_t P, int32_t L, int32_t D, float alpha, float tau,
+                                  int32_t* branch_to_prefix, float* sigma, void* stream) {
+    if (B < 0 || P <= 0 || L <= 0 || D <= 0) return RKSC_ERR_INVALID_ARG;
+    if (B == 0) return RKSC_OK;
+    if (!h_branch || !h_root || !cand_prefix || !branch_to_prefix) return RKSC_ERR_INVALID_ARG;
+    if (!(alpha == alpha) || !(tau == tau)) return RKSC_ERR_INVALID_ARG;
+    if ((int64_t)B * 8 >= ((int64_t)1 << 31)) return RKSC_ERR_UNSUPPORTED;
+    int32_t st = ensure_device(nullptr);
+    if (st != RKSC_OK) return st;
+    cudaError_t e = launch_asks_gate(h_branch, h_root, cand_prefix, B, P, L, D, alpha, tau, branch_to_prefix, sigma,
+                                     static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    return RKSC_OK;
+}
+
+extern "C" RKSC_API int32_t rksc_plan_create(const rksc_layout* layout, const rksc_tables* tables, rksc_plan** out) {
+    if (!layout || !tables || !out) return RKSC_ERR_INVALID_ARG;
+    *out = nullptr;
+    rksc_plan* p = new (std::nothrow) rksc_plan();
+    if (!p) return RKSC_ERR_NOMEM;
+    int ndev = 0;
+    const bool have_dev = (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0);
+    if (!have_dev) cudaGetLastError();
+    int32_t st = RKSC_OK;
+    if (have_dev) {
+        st = ensure_device(&p->device);
+        if (st == RKSC_OK) {
+            int sms = 0;
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, p->device) == cudaSuccess && sms > 0)
+                p->num_sms = sms;
+        }
+    }
+    if (st == RKSC_OK) {
+        try {
+            st = build_host_plan(*layout, *tables, p->num_sms, &p->host);
+        } catch (const std::bad_alloc&) {
+            st = RKSC_ERR_NOMEM;
+        }
+    }
+    if (st == RKSC_OK && have_dev) st = upload_plan(p);
+    if (st != RKSC_OK) {
+        delete p;
+        return st;
+    }
+    *out = p;
+    return RKSC_OK;
+}
+
+extern "C" RKSC_API int32_t rksc_plan_query(const rksc_plan* plan, rksc_plan_info* info) {
+    if (!plan || !info) return RKSC_ERR_INVALID_ARG;
+    const HostPlan& H = plan->host;
+    info->workspace_bytes = H.workspace_bytes;
+    info->mass_elems = H.mass_elems;
+    info->mass_off = H.mass_off.data();
+    info->num_work_items = (int32_t)H.items.size();
+    info->num_partial_rows = H.num_partial_rows;
+    info->unique_kv_tokens = H.unique_kv_tokens;
+    info->duplicated_kv_tokens = H.duplicated_kv_tokens;
+    info->on_device = plan->on_device ? 1 : 0;
+    return RKSC_OK;
+}
+
+extern "C" RKSC_API int32_t rksc_plan_get_item(const rksc_plan* plan, int32_t i, int32_t* out10) {
+    if (!plan || !out10) return RKSC_ERR_INVALID_ARG;
+    const HostPlan& H = plan->host;
+    if (i < 0 || i >= (int32_t)H.items.size()) return RKSC_ERR_INVALID_ARG;
+    const WorkItem& it = H.items[i];
+    out10[0] = it.seg;
+    out10[1] = it.kv_head;
+    out10[2] = it.seg_page_begin;
+    out10[3] = it.num_pages;
+    out10[4] = it.num_tokens;
+    out10[5] = it.sharer_begin - H.seg_sharer_off[it.seg];
+    out10[6] = it.num_sharers;
+    out10[7] = it.part_row_base;
+    out10[8] = it.klass;
+    out10[9] = 0;
+    return RKSC_OK;
+}
+
+extern "C" RKSC_API void rksc_plan_destroy(rksc_plan* plan) {
+    if (!plan) return;
+    if (plan->dev_arena) {
+        int cur = -1;
+        const bool sw = (cudaGetDevice(&cur) == cudaSuccess && cur != plan->device && plan->device >= 0);
+        if (sw) cudaSetDevice(plan->device);
+        cudaFree(plan->dev_arena);
+        if (sw) cudaSetDevice(cur);
+    }
+    delete plan;
+}
+
+extern "C" RKSC_API int32_t rksc_branch_decode_attention(const rksc_plan* plan, const void* q, const void* k_pool,
+                                                const void* v_pool, float* out, float* block_mass, void* workspace,
+                                                size_t workspace_bytes, int32_t* device_status, void* stream) {
+    if (!plan) return RKSC_ERR_INVALID_ARG;
+    const HostPlan& H = plan->host;
+    if (H.B == 0) return RKSC_OK;
+    if (!q || !k_pool || !v_pool || !out) return RKSC_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(k_pool) & 15) ||
+        (reinterpret_cast<uintptr_t>(v_pool) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+        return RKSC_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < H.workspace_bytes || (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return RKSC_ERR_WORKSPACE;
+    if (!plan->on_device) return RKSC_ERR_CUDA;
+    int dev = -1;
+    int32_t st = ensure_device(&dev);
+    if (st != RKSC_OK) return st;
+    if (dev != plan->device) return RKSC_ERR_INVALID_ARG;
+
+    CUtensorMap tm_k, tm_v;
+    st = make_pool_map(H.layout, k_pool, &tm_k);
+    if (st != RKSC_OK) return st;
+    st = make_pool_map(H.layout, v_pool, &tm_v);
+    if (st != RKSC_OK) return st;
+
+    AttnArgs a{};
+    a.plan = plan->dev;
+    a.q = q;
+    a.part_o = static_cast<float*>(workspace);
+    a.part_lse = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + H.ws_lse_offset);
+    a.block_mass = block_mass;
+    a.out = out;
+    a.status = device_status;
+    a.num_items = (int)H.items.size();
+    a.B = H.B;
+    a.Hq = H.layout.num_q_heads;
+    a.Hkv = H.layout.num_kv_heads;
+    a.G = H.G;
+    a.head_dim = H.layout.head_dim;
+    const float scale = H.layout.sm_scale > 0.f ? H.layout.sm_scale : 1.0f / std::sqrt((float)H.layout.head_dim);
+    a.scale_log2 = scale * 1.4426950408889634f;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_seg_attn_warp(tm_k, tm_v, a, s);
+    if (e == cudaSuccess) e = launch_merge(a, s);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    return RKSC_OK;
+}

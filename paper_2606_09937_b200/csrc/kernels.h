@@ -1,0 +1,36 @@
+// Launch prototypes of the kernels (implemented in the .cu files of this directory).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "rksc_internal.h"
+
+namespace rksc {
+
+cudaError_t launch_asks_gate(const float* h_branch, const float* h_root, const int32_t* cand_prefix,
+                             int B, int P, int L, int D, float alpha, float tau,
+                             int32_t* branch_to_prefix, float* sigma, cudaStream_t stream);
+
+struct AttnArgs {
+    DevicePlan plan;
+    const void* q;          // bf16 [B][Hq][d]
+    float* part_o;          // [rows][d]
+    float* part_lse;        // [rows], log2 units
+    float* block_mass;      // may be null; holds log2 masses between the two launches
+    float* out;             // [B][Hq][d]
+    int32_t* status;        // may be null
+    int num_items;
+    int B, Hq, Hkv, G, head_dim;
+    float scale_log2;       // sm_scale * log2(e)
+};
+
+// Sets the kernels' shared-memory attribute for the current device.
+cudaError_t configure_attention_kernels();
+size_t warp_kernel_smem_bytes(int head_dim);
+
+cudaError_t launch_seg_attn_warp(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnArgs& a,
+                                 cudaStream_t stream);
+cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream);
+
+}  // namespace rksc

@@ -1,0 +1,266 @@
+// Host-side integer work: tables from a gate map, table validation, sharing groups,
+// KV chunking, workspace and block-mass layout.  No CUDA calls in this file.
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <numeric>
+
+#include "rksc_internal.h"
+
+namespace rksc {
+
+namespace {
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+bool csr_ok(const int32_t* off, int n) {
+    if (off[0] != 0) return false;
+    for (int i = 0; i < n; ++i)
+        if (off[i + 1] < off[i]) return false;
+    return true;
+}
+
+}  // namespace
+
+int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms, HostPlan* hp) {
+    if (L.num_q_heads <= 0 || L.num_kv_heads <= 0 || L.num_pool_blocks <= 0) return RKSC_ERR_INVALID_ARG;
+    if (L.num_q_heads % L.num_kv_heads != 0) return RKSC_ERR_INVALID_ARG;
+    if (L.block_size != kBlock) return RKSC_ERR_UNSUPPORTED;
+    if (L.head_dim != 64 && L.head_dim != 128) return RKSC_ERR_UNSUPPORTED;
+    const int G = L.num_q_heads / L.num_kv_heads;
+    if (G > kMaxRowsPerItem) return RKSC_ERR_UNSUPPORTED;
+    if ((int64_t)L.num_pool_blocks * L.num_kv_heads * kBlock >= (int64_t)1 << 31) return RKSC_ERR_UNSUPPORTED;
+    if (t.num_branches < 0 || t.num_segments < 0) return RKSC_ERR_INVALID_ARG;
+    if (!t.seg_block_off || !t.br_seg_off) return RKSC_ERR_INVALID_ARG;
+    const int B = t.num_branches, S = t.num_segments;
+    if (S > 0 && !t.seg_num_tokens) return RKSC_ERR_INVALID_ARG;
+    if (!csr_ok(t.seg_block_off, S) || !csr_ok(t.br_seg_off, B)) return RKSC_ERR_BAD_TABLE;
+    const int total_pages = t.seg_block_off[S];
+    const int total_refs = t.br_seg_off[B];
+    if (total_pages > 0 && !t.seg_blocks) return RKSC_ERR_INVALID_ARG;
+    if (total_refs > 0 && !t.br_segs) return RKSC_ERR_INVALID_ARG;
+
+    for (int s = 0; s < S; ++s) {
+        const int np = t.seg_block_off[s + 1] - t.seg_block_off[s];
+        const int nt = t.seg_num_tokens[s];
+        if (nt < 0 || np != ceil_div(nt, kBlock)) return RKSC_ERR_BAD_TABLE;
+    }
+    for (int i = 0; i < total_pages; ++i)
+        if (t.seg_blocks[i] < 0 || t.seg_blocks[i] >= L.num_pool_blocks) return RKSC_ERR_BAD_TABLE;
+    for (int i = 0; i < total_refs; ++i)
+        if (t.br_segs[i] < 0 || t.br_segs[i] >= S) return RKSC_ERR_BAD_TABLE;
+
+    HostPlan& P = *hp;
+    P = HostPlan{};
+    P.layout = L;
+    P.B = B;
+    P.S = S;
+    P.G = G;
+    P.seg_block_off.assign(t.seg_block_off, t.seg_block_off + S + 1);
+    P.seg_blocks.assign(t.seg_blocks, t.seg_blocks + total_pages);
+    P.seg_num_tokens.assign(t.seg_num_tokens, t.seg_num_tokens + S);
+
+    // logical block counts and mass offsets
+    P.br_nblk.assign(B, 0);
+    P.mass_off.assign(B + 1, 0);
+    for (int b = 0; b < B; ++b) {
+        int64_t n = 0, tok = 0;
+        for (int i = t.br_seg_off[b]; i < t.br_seg_off[b + 1]; ++i) {
+            const int s = t.br_segs[i];
+            n += P.seg_block_off[s + 1] - P.seg_block_off[s];
+            tok += P.seg_num_tokens[s];
+        }
+        if (n >= ((int64_t)1 << 31)) return RKSC_ERR_UNSUPPORTED;
+        P.br_nblk[b] = (int32_t)n;
+        P.mass_off[b + 1] = P.mass_off[b] + n;
+        P.duplicated_kv_tokens += tok;
+    }
+    P.mass_elems = P.mass_off[B] * L.num_q_heads;
+
+    // sharing groups: for every segment the ascending list of (branch, mass position)
+    P.seg_sharer_off.assign(S + 1, 0);
+    for (int i = 0; i < total_refs; ++i) P.seg_sharer_off[t.br_segs[i] + 1]++;
+    for (int s = 0; s < S; ++s) P.seg_sharer_off[s + 1] += P.seg_sharer_off[s];
+    P.sharers.resize(total_refs);
+    {
+        std::vector<int32_t> fill(P.seg_sharer_off.begin(), P.seg_sharer_off.end() - 1);
+        for (int b = 0; b < B; ++b) {
+            int64_t loff = 0;
+            for (int i = t.br_seg_off[b]; i < t.br_seg_off[b + 1]; ++i) {
+                const int s = t.br_segs[i];
+                Sharer sh;
+                sh.branch = b;
+                sh.nblk = P.br_nblk[b];
+                sh.mass_base = P.mass_off[b] * L.num_q_heads + loff;
+                P.sharers[fill[s]++] = sh;
+                loff += P.seg_block_off[s + 1] - P.seg_block_off[s];
+            }
+        }
+    }
+
+    // chunking: sharer blocks of at most kMaxRowsPerItem rows, KV chunks sized so that the
+    // launch fills the device while partial results stay a few percent of the KV bytes read
+    const int per_block = std::max(1, kMaxRowsPerItem / G);
+    int64_t total_units = 0;  // page-heads over all (segment, sharer block)
+    for (int s = 0; s < S; ++s) {
+        const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
+        const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
+        if (ns == 0 || np == 0) continue;
+        P.unique_kv_tokens += P.seg_num_tokens[s];
+        total_units += (int64_t)np * L.num_kv_heads * ceil_div(ns, per_block);
+    }
+    const int slots = std::max(1, num_sms) * 2;
+    const int kMinChunk = 8;
+    const int upper = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, total_units / slots));
+
+    int64_t rows_total = 0;
+    for (int s = 0; s < S; ++s) {
+        const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
+        const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
+        if (ns == 0 || np == 0) continue;
+        const int nsb = ceil_div(ns, per_block);
+        for (int sb = 0; sb < nsb; ++sb) {
+            // balanced split of the sharers
+            const int sh_lo = (int)((int64_t)ns * sb / nsb), sh_hi = (int)((int64_t)ns * (sb + 1) / nsb);
+            const int rows = (sh_hi - sh_lo) * G;
+            const int want = std::min(upper, std::max(kMinChunk, 2 * rows));
+            const int nch = ceil_div(np, want);
+            for (int c = 0; c < nch; ++c) {
+                const int p_lo = (int)((int64_t)np * c / nch), p_hi = (int)((int64_t)np * (c + 1) / nch);
+                const int tok_lo = p_lo * kBlock;
+                const int tok_hi = std::min(P.seg_num_tokens[s], p_hi * kBlock);
+                for (int h = 0; h < L.num_kv_heads; ++h) {
+                    WorkItem it{};
+                    it.seg = s;
+                    it.kv_head = h;
+                    it.page_begin = P.seg_block_off[s] + p_lo;
+                    it.num_pages = p_hi - p_lo;
+                    it.num_tokens = tok_hi - tok_lo;
+                    it.sharer_begin = P.seg_sharer_off[s] + sh_lo;
+                    it.num_sharers = sh_hi - sh_lo;
+                    it.part_row_base = 0;  // set after sorting
+                    it.seg_page_begin = p_lo;
+                    it.klass = 0;
+                    P.items.push_back(it);
+                    rows_total += rows;
+                }
+            }
+        }
+    }
+    if (rows_total >= ((int64_t)1 << 31)) return RKSC_ERR_UNSUPPORTED;
+
+    // longest first, so the hardware block scheduler packs the tail with short items
+    std::stable_sort(P.items.begin(), P.items.end(), [G](const WorkItem& a, const WorkItem& b) {
+        const int64_t ca = (int64_t)a.num_pages * (3 + ceil_div(a.num_sharers * G, 16));
+        const int64_t cb = (int64_t)b.num_pages * (3 + ceil_div(b.num_sharers * G, 16));
+        return ca > cb;
+    });
+    int32_t row = 0;
+    for (auto& it : P.items) {
+        it.part_row_base = row;
+        row += it.num_sharers * G;
+    }
+    P.num_partial_rows = row;
+
+    // merge lists: for every (branch, kv head) the partial rows (of head-in-group 0) to combine
+    const int nkeys = B * L.num_kv_heads;
+    P.merge_off.assign(nkeys + 1, 0);
+    for (const auto& it : P.items)
+        for (int i = 0; i < it.num_sharers; ++i)
+            P.merge_off[P.sharers[it.sharer_begin + i].branch * L.num_kv_heads + it.kv_head + 1]++;
+    for (int k = 0; k < nkeys; ++k) P.merge_off[k + 1] += P.merge_off[k];
+    P.merge_rows.resize(P.merge_off[nkeys]);
+    {
+        std::vector<int32_t> fill(P.merge_off.begin(), P.merge_off.end() - 1);
+        for (const auto& it : P.items)
+            for (int i = 0; i < it.num_sharers; ++i) {
+                const int key = P.sharers[it.sharer_begin + i].branch * L.num_kv_heads + it.kv_head;
+                P.merge_rows[fill[key]++] = it.part_row_base + i * G;
+            }
+    }
+
+    // workspace: partial outputs [rows][d] fp32, then partial log2-sum-exp [rows] fp32
+    const size_t o_bytes = ((size_t)P.num_partial_rows * L.head_dim * sizeof(float) + 255) / 256 * 256;
+    P.ws_lse_offset = o_bytes;
+    P.workspace_bytes = o_bytes + ((size_t)P.num_partial_rows * sizeof(float) + 255) / 256 * 256;
+    if (P.workspace_bytes == 0) P.workspace_bytes = 256;
+    return RKSC_OK;
+}
+
+}  // namespace rksc
+
+// ---------------------------------------------------------------------------------------------
+// C ABI: tables from a gate map
+// ---------------------------------------------------------------------------------------------
+
+extern "C" RKSC_API int32_t rksc_tables_from_gate(int32_t B, int32_t P, const int32_t* map,
+                                         const int32_t* shared_off, const int32_t* shared_pages, const int32_t* shared_ntok,
+                                         const int32_t* priv_off, const int32_t* priv_pages, const int32_t* priv_ntok,
+                                         const int32_t* sfx_off, const int32_t* sfx_pages, const int32_t* sfx_ntok,
+                                         rksc_tables* out) {
+    if (!out) return RKSC_ERR_INVALID_ARG;
+    std::memset(out, 0, sizeof(*out));
+    if (B < 0 || P < 0) return RKSC_ERR_INVALID_ARG;
+    if (B > 0 && (!map || !priv_off || !priv_ntok || !sfx_off || !sfx_ntok)) return RKSC_ERR_INVALID_ARG;
+    if (P > 0 && (!shared_off || !shared_ntok)) return RKSC_ERR_INVALID_ARG;
+    for (int b = 0; b < B; ++b)
+        if (map[b] >= P) return RKSC_ERR_INVALID_ARG;
+
+    std::vector<int32_t> shared_seg(P > 0 ? P : 1, -1);
+    std::vector<int32_t> seg_off{0}, blocks, ntok, br_segs((size_t)2 * B);
+    try {
+        auto add = [&](const int32_t* off, const int32_t* pages, const int32_t* nt, int i) {
+            for (int k = off[i]; k < off[i + 1]; ++k) blocks.push_back(pages[k]);
+            seg_off.push_back((int32_t)blocks.size());
+            ntok.push_back(nt[i]);
+            return (int32_t)ntok.size() - 1;
+        };
+        std::vector<char> has(P > 0 ? P : 1, 0);
+        for (int b = 0; b < B; ++b)
+            if (map[b] >= 0) has[map[b]] = 1;
+        for (int r = 0; r < P; ++r)
+            if (has[r]) shared_seg[r] = add(shared_off, shared_pages, shared_ntok, r);
+        for (int b = 0; b < B; ++b)
+            if (map[b] < 0) br_segs[2 * b] = add(priv_off, priv_pages, priv_ntok, b);
+            else br_segs[2 * b] = shared_seg[map[b]];
+        for (int b = 0; b < B; ++b) br_segs[2 * b + 1] = add(sfx_off, sfx_pages, sfx_ntok, b);
+    } catch (const std::bad_alloc&) {
+        return RKSC_ERR_NOMEM;
+    }
+    const int S = (int)ntok.size();
+    auto dup = [](const std::vector<int32_t>& v, size_t n) -> int32_t* {
+        int32_t* p = (int32_t*)std::malloc(std::max<size_t>(1, n) * sizeof(int32_t));
+        if (p && n) std::memcpy(p, v.data(), n * sizeof(int32_t));
+        return p;
+    };
+    std::vector<int32_t> br_off(B + 1);
+    for (int b = 0; b <= B; ++b) br_off[b] = 2 * b;
+    int32_t* a0 = dup(seg_off, S + 1);
+    int32_t* a1 = dup(blocks, blocks.size());
+    int32_t* a2 = dup(ntok, S);
+    int32_t* a3 = dup(br_off, B + 1);
+    int32_t* a4 = dup(br_segs, (size_t)2 * B);
+    if (!a0 || !a1 || !a2 || !a3 || !a4) {
+        std::free(a0); std::free(a1); std::free(a2); std::free(a3); std::free(a4);
+        return RKSC_ERR_NOMEM;
+    }
+    out->num_branches = B;
+    out->num_segments = S;
+    out->seg_block_off = a0;
+    out->seg_blocks = a1;
+    out->seg_num_tokens = a2;
+    out->br_seg_off = a3;
+    out->br_segs = a4;
+    return RKSC_OK;
+}
+
+extern "C" RKSC_API void rksc_tables_free(rksc_tables* t) {
+    if (!t) return;
+    std::free((void*)t->seg_block_off);
+    std::free((void*)t->seg_blocks);
+    std::free((void*)t->seg_num_tokens);
+    std::free((void*)t->br_seg_off);
+    std::free((void*)t->br_segs);
+    std::memset(t, 0, sizeof(*t));
+}

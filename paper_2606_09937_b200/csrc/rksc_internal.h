@@ -1,0 +1,82 @@
+// Internal structures shared by the host-side plan and the kernels.
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "rksc.h"
+
+namespace rksc {
+
+constexpr int kBlock = RKSC_BLOCK_SIZE;     // tokens per KV page
+constexpr int kMaxRowsPerItem = 64;         // stacked query rows one warp-MMA work item handles
+constexpr int kMaxPagesPerItem = 512;       // page ids a CTA caches in shared memory
+constexpr int kWarpKernelThreads = 128;
+constexpr int kWarpKernelSlots = 12;        // (K page + V page) ring slots per CTA
+
+// One CTA's work: a chunk of one segment's pages for one KV head and a block of the
+// segment's sharers.  Stacked rows = num_sharers * G, row r <-> (sharer r / G, head r % G).
+struct WorkItem {
+    int32_t seg;
+    int32_t kv_head;
+    int32_t page_begin;      // absolute index into the flattened page-id array
+    int32_t num_pages;
+    int32_t num_tokens;      // valid tokens in this chunk
+    int32_t sharer_begin;    // absolute index into the sharer array
+    int32_t num_sharers;
+    int32_t part_row_base;   // first row of this item's partial results
+    int32_t seg_page_begin;  // index of the first page within its segment
+    int32_t klass;           // 0: warp-MMA kernel
+};
+
+// A (segment, branch) incidence: where the branch's masses of this segment start.
+struct Sharer {
+    int32_t branch;
+    int32_t nblk;            // logical blocks of the branch = stride between heads in block_mass
+    int64_t mass_base;       // mass_off[branch] * Hq + logical block offset of the segment
+};
+
+struct DevicePlan {
+    const WorkItem* items = nullptr;
+    const int32_t* seg_blocks = nullptr;
+    const Sharer* sharers = nullptr;
+    const int32_t* merge_off = nullptr;   // [B*Hkv + 1]
+    const int32_t* merge_rows = nullptr;  // partial row of head-in-group 0 for each part
+    const int64_t* mass_off = nullptr;    // [B+1]
+    const int32_t* br_nblk = nullptr;     // [B]
+};
+
+struct HostPlan {
+    rksc_layout layout{};
+    int32_t B = 0, S = 0, G = 1;
+    std::vector<int32_t> seg_blocks;      // flattened page ids of the segments that have sharers... all segments
+    std::vector<int32_t> seg_block_off;
+    std::vector<int32_t> seg_num_tokens;
+    std::vector<WorkItem> items;
+    std::vector<Sharer> sharers;
+    std::vector<int32_t> seg_sharer_off;  // [S+1]
+    std::vector<int32_t> merge_off;
+    std::vector<int32_t> merge_rows;
+    std::vector<int64_t> mass_off;        // [B+1]
+    std::vector<int32_t> br_nblk;         // [B]
+    int64_t mass_elems = 0;
+    int32_t num_partial_rows = 0;
+    int64_t unique_kv_tokens = 0, duplicated_kv_tokens = 0;
+    size_t workspace_bytes = 0;
+    size_t ws_lse_offset = 0;             // byte offset of the lse array inside the workspace
+};
+
+// Builds every host list from validated tables.  num_sms sizes the KV chunks.
+int32_t build_host_plan(const rksc_layout& layout, const rksc_tables& t, int num_sms, HostPlan* hp);
+
+}  // namespace rksc
+
+struct rksc_plan {
+    rksc::HostPlan host;
+    rksc::DevicePlan dev;
+    void* dev_arena = nullptr;
+    int device = -1;
+    int num_sms = 148;
+    bool on_device = false;
+};

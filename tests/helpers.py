@@ -81,3 +81,34 @@ def check_attention(out, masses, ref_out, ref_masses, branches=None):
         assert max_mass <= MASS_ATOL, f"mass max-abs {max_mass}"
         assert max_sum <= MASS_SUM_ATOL, f"mass sum {max_sum}"
     return {"max_abs": max_abs, "max_rel": max_rel, "max_mass": max_mass, "max_mass_sum": max_sum}
+
+
+# ---------------------------------------------------------------------------------------
+# CUDA path (through the C ABI binding)
+# ---------------------------------------------------------------------------------------
+
+def cuda_attention(w, tables=None, want_mass=True, pools=None):
+    """Run the library on a workload; returns (out numpy, masses list, plan)."""
+    import torch
+    import paper_2606_09937_b200 as rk
+    t = tables if tables is not None else w.tables
+    plan = rk.rksc_plan_create(w.layout, t)
+    dev = torch.device("cuda:0")
+    if pools is None:
+        pools = (w.k_pool.to(dev), w.v_pool.to(dev))
+    q = w.q.to(dev)
+    out, mass, status = rk.rksc_branch_decode_attention(plan, q, pools[0], pools[1], want_mass=want_mass)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    masses = rk.split_block_mass(plan, mass) if want_mass else None
+    return out.cpu().numpy(), masses, plan
+
+
+def cuda_gate(g):
+    import torch
+    import paper_2606_09937_b200 as rk
+    dev = torch.device("cuda:0")
+    m, s = rk.rksc_asks_gate(g.h_branch.to(dev), g.h_root.to(dev),
+                             torch.from_numpy(g.cand_prefix).to(dev), g.alpha, g.tau)
+    torch.cuda.synchronize()
+    return m.cpu().numpy(), s.cpu().numpy()

@@ -1,0 +1,111 @@
+"""CUDA path vs the fp64 oracle, element by element, on small and edge-case inputs."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import workloads
+from helpers import (check_attention, cuda_attention, cuda_gate, oracle_attention, oracle_gate,
+                     oracle_tables_from_map)
+
+pytestmark = pytest.mark.gpu
+
+
+def _parity(w, tables=None):
+    ref_out, ref_m = oracle_attention(w, tables)
+    out, m, plan = cuda_attention(w, tables)
+    return check_attention(out, m, ref_out, ref_m), plan
+
+
+def test_tiny_as_stated():
+    w = workloads.make_tiny()
+    err, plan = _parity(w)
+    assert plan.unique_kv_tokens == 384 and plan.duplicated_kv_tokens == 1152
+
+
+def test_tiny_end_to_end_gate_tables_attention():
+    import paper_2606_09937_b200 as rk
+    w = workloads.make_tiny()
+    m_ref, s_ref = oracle_gate(w.gate)
+    m, s = cuda_gate(w.gate)
+    assert m.tolist() == m_ref.tolist() == workloads.make_tiny_gate_tables()["map"]
+    assert np.abs(s - s_ref).max() < 1e-5
+    f = w.flat
+    t = rk.rksc_tables_from_gate(m, f.num_prefixes, f.shared_off, f.shared_pages, f.shared_ntok,
+                                 f.priv_off, f.priv_pages, f.priv_ntok, f.sfx_off, f.sfx_pages, f.sfx_ntok)
+    t_ref = oracle_tables_from_map(w, m_ref)
+    for k, v in t.as_dict().items():
+        assert np.array_equal(v, t_ref[k]), k
+    _parity(w, t_ref)
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 64), (28, 4, 128), (32, 8, 128), (4, 4, 128), (16, 1, 64)])
+def test_ragged_segments(hq, hkv, d):
+    # partial pages, one-token segments, empty segment, empty branch, shared + private mix
+    seg_ntok = [37, 5, 16, 1, 0, 100, 17]
+    br = [[0, 1], [0, 2], [3], [0, 4, 5], [], [5, 6], [0, 5, 6]]
+    w = workloads.make_from_segments("ragged", hq, hkv, d, seg_ntok, br, seed=11)
+    _parity(w)
+
+
+@pytest.mark.parametrize("sharers,G", [(1, 1), (3, 5), (9, 7), (16, 4), (17, 4), (4, 16), (33, 2), (70, 1)])
+def test_row_counts_around_tile_edges(sharers, G):
+    # stacked rows = sharers * G: 1, 15, 63, 64, 68 (two sharer blocks), 64, 66, 70
+    hkv = 2
+    w = workloads.make_from_segments("rows", G * hkv, hkv, 128, [200] + [19] * sharers,
+                                     [[0, 1 + b] for b in range(sharers)], seed=12 + sharers)
+    _parity(w)
+
+
+def test_long_segment_many_chunks_and_custom_scale():
+    w = workloads.make_from_segments("long", 8, 2, 128, [5000, 33, 700], [[0, 1], [0, 2], [0]], seed=13,
+                                     sm_scale=0.11)
+    err, plan = _parity(w)
+    assert plan.num_work_items > 8
+
+
+def test_tot_small():
+    w = workloads.make_tot(root_tokens=300, level_tokens=50)
+    _parity(w)
+
+
+def test_sharp_softmax_large_values():
+    # queries scaled x6: near one-hot attention, stresses the running-max rescaling and the abs tolerance
+    w = workloads.make_from_segments("sharp", 8, 2, 64, [300, 40], [[0, 1], [0]], seed=14, q_gain=6.0)
+    _parity(w)
+
+
+def test_without_mass_output():
+    w = workloads.make_tiny()
+    ref_out, _ = oracle_attention(w)
+    out, _, _ = cuda_attention(w, want_mass=False)
+    check_attention(out, None, ref_out, None)
+
+
+def test_holes():
+    w = workloads.make_long_context(prefix=1500, suffix=70, branches=5, num_q_heads=8, num_kv_heads=2, head_dim=128)
+    _, m = oracle_attention(w)
+    npg = int(w.tables.seg_block_off[1])
+    scores = sum(mb[:, :npg].sum(axis=0) for mb in m)
+    h = workloads.punch_holes(w, 0, workloads.lowest_mass_pages(scores, 0.2))
+    _parity(h)
+
+
+def test_gate_edge_cases():
+    import torch
+    # odd D (scalar path), L not a multiple of anything, several roots, zero-norm layer
+    g = workloads.make_gate_inputs([2, 0, 1, 1, 2, 0, 0], 3, 5, 77, [0.0, 0.2, 0.75, 0.1, 2.0, 0.3, float("inf")],
+                                   alpha=1.5, tau=0.82, seed=21)
+    g.h_branch[3, 2] = 0
+    m_ref, s_ref = oracle_gate(g)
+    m, s = cuda_gate(g)
+    assert np.abs(s - s_ref).max() < 1e-5 and m.tolist() == m_ref.tolist()
+    for L, D in ((1, 4), (33, 256), (40, 4096), (64, 100)):
+        B = 9
+        g = workloads.make_gate_inputs([b % 2 for b in range(B)], 2, L, D,
+                                       [0.05 * b for b in range(B)], alpha=0.5, tau=0.9, seed=22 + L)
+        m_ref, s_ref = oracle_gate(g)
+        m, s = cuda_gate(g)
+        assert np.abs(s - s_ref).max() < 1e-5
+        clear = np.abs(s_ref - np.float32(0.9)) > 1e-3
+        assert np.array_equal(m[clear], m_ref[clear])
