@@ -1,0 +1,476 @@
+#!/usr/bin/env python
+"""Benchmark of the ASKS hot path on B200: gate -> tables -> plan -> shared-prefix decode attention.
+
+One "step" is one pass of the whole path over one batch of synthetic input that is already in
+HBM: the gate kernel, the map's copy to the host, table and plan construction, and the
+branch-decode attention (segment kernel + merge).  The metric is unique-KV bytes per second:
+the valid tokens of the distinct KV segments the batch references, times bytes per token,
+divided by the step time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints one JSON line (rank 0).  With N > 1 (launched by torchrun) every rank runs its own
+batch (seed + rank): the path shards by problem, there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "branch_decode_attention_unique_kv_throughput"
+UNIT = "TB/s"
+NOMINAL_HBM_TBPS = 8.0       # the figure the target (>= 70 %) is stated against
+FALLBACK_HBM_GBS = 6650.0    # used only when MEASURED_PEAKS.json is absent
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the segment kernel, from the ncu
+# capture summarised under profiles/ (None until a capture of that workload exists).
+NCU_TRAFFIC_BYTES = {}
+
+WORKLOAD_LABEL = {
+    "tiny": "configs[0] tiny: 8q/2kv d64, 4 branches, prefix 256 + suffix 32",
+    "qwen_layer": "configs[1] Qwen-7B-shaped layer: 28q/4kv d128, 4 branches, prefix 2048 + suffix 512",
+    "tot": "configs[2] Tree-of-Thoughts (4,3): 64 leaves, root 1024 + 3 x 256, 32q/8kv d128",
+    "batched_serving": "configs[3] batched serving: 32 problems x 8 branches, prefix U[512,4096], "
+                       "suffix U[128,1024], 28q/4kv d128, 30% of branches below tau",
+    "long_context": "configs[4] long context with eviction holes: 16 branches, prefix 32768 (20% of pages "
+                    "evicted) + suffix 2048, 32q/8kv d128",
+}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="batched_serving", choices=list(WORKLOAD_LABEL))
+    ap.add_argument("--cpu-sample-branches", type=int, default=96)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the per-config attention-only table")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks sampling during the timed region
+# ----------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------
+# workload set-up
+# ----------------------------------------------------------------------------------------------
+
+def load_workload(name: str, seed_shift: int = 0):
+    import workloads
+    base = {"tiny": 0, "qwen_layer": 1, "tot": 2, "batched_serving": 3, "long_context": 4}[name]
+    return workloads.make_config(name, seed=workloads.generators.SEED_BASE + base + 1000 * seed_shift)
+
+
+class DeviceBatch:
+    """A workload resident in HBM plus the reusable output buffers."""
+
+    def __init__(self, w, dev):
+        import torch
+        self.w = w
+        self.dev = dev
+        self.q = w.q.to(dev)
+        self.k_pool = w.k_pool.to(dev)
+        self.v_pool = w.v_pool.to(dev)
+        self.has_gate = w.gate is not None and w.flat is not None
+        if w.gate is not None:
+            self.h_branch = w.gate.h_branch.to(dev)
+            self.h_root = w.gate.h_root.to(dev)
+            self.cand = torch.from_numpy(w.gate.cand_prefix).to(dev)
+            self.map_dev = torch.empty(self.q.shape[0], dtype=torch.int32, device=dev)
+            self.sigma_dev = torch.empty(self.q.shape[0], dtype=torch.float32, device=dev)
+            self.map_host = torch.empty(self.q.shape[0], dtype=torch.int32).pin_memory()
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.out = torch.empty(tuple(self.q.shape), dtype=torch.float32, device=dev)
+        self.mass = None
+        self.workspace = None
+        self.tables = w.tables
+
+    def ensure_buffers(self, plan):
+        import torch
+        if self.mass is None or self.mass.numel() < max(plan.mass_elems, 1):
+            self.mass = torch.empty(max(plan.mass_elems, 1), dtype=torch.float32, device=self.dev)
+        if self.workspace is None or self.workspace.numel() < plan.workspace_bytes:
+            self.workspace = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device=self.dev)
+
+
+def run_step(rk, batch: DeviceBatch, seg_events=None):
+    """One pass of the hot path.  Returns the plan (for byte counts).  3 kernel launches (2 without a gate)."""
+    w = batch.w
+    launches = 0
+    if batch.has_gate:
+        g, f = w.gate, w.flat
+        rk.rksc_asks_gate(batch.h_branch, batch.h_root, batch.cand, g.alpha, g.tau,
+                          branch_to_prefix=batch.map_dev, sigma=batch.sigma_dev)
+        launches += 1
+        batch.map_host.copy_(batch.map_dev, non_blocking=False)   # the host needs the map to build tables
+        tables = rk.rksc_tables_from_gate(batch.map_host.numpy(), f.num_prefixes,
+                                          f.shared_off, f.shared_pages, f.shared_ntok,
+                                          f.priv_off, f.priv_pages, f.priv_ntok,
+                                          f.sfx_off, f.sfx_pages, f.sfx_ntok)
+    else:
+        tables = batch.tables
+    plan = rk.rksc_plan_create(w.layout, tables)
+    batch.ensure_buffers(plan)
+    kw = dict(out=batch.out, block_mass=batch.mass, workspace=batch.workspace, device_status=batch.status)
+    if seg_events is None:
+        rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, **kw)
+    else:
+        seg_events[0].record()
+        rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=1, **kw)
+        seg_events[1].record()
+        rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=2, **kw)
+    launches += 2
+    return plan, launches
+
+
+def attention_only_times(rk, batch: DeviceBatch, plan, iters: int, flush):
+    """Per-iteration CUDA-event times (ms) of the attention call alone, L2 flushed before each."""
+    import torch
+    kw = dict(out=batch.out, block_mass=batch.mass, workspace=batch.workspace, device_status=batch.status)
+    times = []
+    for _ in range(iters):
+        flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, **kw)
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+    return times
+
+
+def algorithmic_bytes(plan, layout):
+    """Bytes the segment kernel has to move by definition: unique KV + queries + page ids + block masses."""
+    bpt = 2 * layout.num_kv_heads * layout.head_dim * 2
+    kv = plan.unique_kv_tokens * bpt
+    qb = plan.num_branches * layout.num_q_heads * layout.head_dim * 2
+    tables = 4 * int(plan.tables.seg_block_off[-1])
+    mass = 4 * plan.mass_elems
+    return kv, kv + qb + tables + mass
+
+
+# ----------------------------------------------------------------------------------------------
+# the oracle as CPU baseline / reference arm
+# ----------------------------------------------------------------------------------------------
+
+def oracle_pass(w, sample_branches: int):
+    """The oracle on a bounded sample (the first branches of the batch).  Returns (seconds, unique bytes, cores)."""
+    import oracle
+    import workloads
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    L = w.layout
+    q = oracle.to_f32_numpy(w.q)
+    kp = oracle.to_f32_numpy(w.k_pool)
+    vp = oracle.to_f32_numpy(w.v_pool)
+    t0 = time.perf_counter()
+    if w.gate is not None and w.flat is not None:
+        g, f = w.gate, w.flat
+        m, _ = oracle.asks_gate(g.h_branch.numpy(), g.h_root.numpy(), g.cand_prefix, g.alpha, g.tau)
+        t = oracle.tables_from_gate(m, f.num_prefixes, f.shared_off, f.shared_pages, f.shared_ntok,
+                                    f.priv_off, f.priv_pages, f.priv_ntok, f.sfx_off, f.sfx_pages, f.sfx_ntok)
+    else:
+        tt = w.tables
+        t = {k: getattr(tt, k) for k in ("seg_block_off", "seg_blocks", "seg_num_tokens", "br_seg_off", "br_segs")}
+    B = len(t["br_seg_off"]) - 1
+    nb = min(B, max(1, sample_branches))
+    oracle.branch_decode_attention(L.num_q_heads, L.num_kv_heads, L.head_dim, L.sm_scale,
+                                   t["seg_block_off"], t["seg_blocks"], t["seg_num_tokens"],
+                                   t["br_seg_off"], t["br_segs"], q, kp, vp, branches=range(nb))
+    dt = time.perf_counter() - t0
+    segs = np.unique(t["br_segs"][: t["br_seg_off"][nb]])
+    ubytes = int(sum(int(t["seg_num_tokens"][s]) for s in segs)) * L.bytes_per_token
+    return dt, ubytes, cores, nb, B
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = load_workload(args.workload)
+    times, ub = [], 0
+    nb = B = 0
+    cores = 1
+    for i in range(args.warmup + args.steps):
+        dt, ub, cores, nb, B = oracle_pass(w, args.cpu_sample_branches)
+        if i >= args.warmup:
+            times.append(dt)
+    t = sum(times) / len(times)
+    val = ub / t / 1e12
+    sample = f"first {nb} of {B} branches of the batch (gate over all branches, attention over the sample)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD_LABEL[args.workload], "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import paper_2606_09937_b200 as rk
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    rk.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = load_workload(args.workload, seed_shift=rank)
+    batch = DeviceBatch(w, dev)
+    if w.name == "long_context":
+        punch_long_context(rk, batch)
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    flush_buf = torch.empty(max(2 * l2_bytes, 256 << 20), dtype=torch.uint8, device=dev)
+
+    def flush():
+        flush_buf.fill_(1)
+
+    plan = None
+    for _ in range(max(args.warmup, 3)):
+        plan, _ = run_step(rk, batch)
+    torch.cuda.synchronize()
+    assert int(batch.status.item()) == 0, "a kernel reported a device-side timeout"
+    kv_bytes, alg_bytes = algorithmic_bytes(plan, w.layout)
+    small = kv_bytes < 2 * l2_bytes   # then L2 must be flushed between timed iterations
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    seg_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    step_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches = 0
+    barrier()
+    t_wall0 = time.perf_counter()
+    for i in range(args.steps):
+        if small:
+            flush()
+        step_ev[i][0].record()
+        plan, n = run_step(rk, batch, seg_events=seg_ev[i])
+        step_ev[i][1].record()
+        launches += n
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop() if rank == 0 else None
+    step_ms = [a.elapsed_time(b) for a, b in step_ev]
+    seg_ms = [a.elapsed_time(b) for a, b in seg_ev]
+    total_ms = sum(step_ms)           # device time of exactly K steps (flushes excluded)
+    tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    total_ms_max = float(tt.item())
+    assert int(batch.status.item()) == 0, "a kernel reported a device-side timeout"
+
+    value = world * kv_bytes * args.steps / (total_ms_max * 1e-3) / 1e12
+    peak_gbs, peak_kind = measured_peak_gbs()
+    seg_avg_ms = sum(seg_ms) / len(seg_ms)
+    achieved = alg_bytes / (seg_avg_ms * 1e-3) / 1e9
+    B = w.num_branches
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": WORKLOAD_LABEL[args.workload],
+            "step": "gate kernel + map D2H + tables + plan + attention (segment kernel + merge)",
+            "unique_kv_bytes": kv_bytes, "branches": B, "work_items": plan.num_work_items,
+            "l2": ("inputs larger than L2 (unique KV %.0f MB vs L2 %.0f MB)" % (kv_bytes / 1e6, l2_bytes / 1e6))
+            if not small else "L2 flushed (write of 2x L2) before every timed step",
+            "sharding": "one batch per rank (seed + rank), no data-path collective",
+        },
+        "branch_steps_per_s": world * B * args.steps / (total_ms_max * 1e-3),
+        "pct_of_8tbps": 100.0 * value / world / NOMINAL_HBM_TBPS,
+        "pct_of_measured_copy_peak": 100.0 * value * 1e3 / world / peak_gbs,
+        "wall_ms_per_step": t_wall * 1e3 / args.steps,
+        "gpu_launches": launches,
+        "roofline": {
+            "kernel": "seg_attn_warp_kernel", "bound": "hbm", "achieved": achieved, "peak": peak_gbs,
+            "unit": "GB/s", "frac": achieved / peak_gbs, "peak_source": peak_kind,
+            "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": seg_avg_ms,
+            "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+        },
+        "clocks": clocks,
+    }
+
+    if rank == 0 and world == 1:
+        att = attention_only_times(rk, batch, plan, max(10, args.steps), flush)
+        med = statistics.median(att)
+        line["attention_only"] = {
+            "what": "one rksc_branch_decode_attention call (segment kernel + merge), plan prebuilt, cold L2",
+            "ms_median": med, "ms_min": min(att), "tbps_unique_kv": kv_bytes / (med * 1e-3) / 1e12,
+            "pct_of_8tbps": 100.0 * kv_bytes / (med * 1e-3) / 1e12 / NOMINAL_HBM_TBPS,
+            "pct_of_measured_copy_peak": 100.0 * kv_bytes / (med * 1e-3) / 1e9 / peak_gbs,
+            "branch_steps_per_s": B / (med * 1e-3),
+        }
+        if not args.no_sweep:
+            line["configs"] = sweep_configs(rk, dev, flush, peak_gbs, skip=args.workload, cached=(args.workload, line))
+        if not args.no_cpu_baseline:
+            dt, ub, cores, nb, Bt = oracle_pass(w, args.cpu_sample_branches)
+            line["cpu_baseline"] = {
+                "value": ub / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"first {nb} of {Bt} branches of the batch (gate over all, attention over the sample), "
+                          f"{dt:.1f} s", "seconds": dt}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def punch_long_context(rk, batch: DeviceBatch):
+    """Config 5: evict the 20 % of prefix pages with the lowest mass of a prior full-table step (computed on the GPU)."""
+    import torch
+    import workloads
+    w = batch.w
+    plan = rk.rksc_plan_create(w.layout, w.tables)
+    batch.ensure_buffers(plan)
+    _, mass, _ = rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, out=batch.out,
+                                                 block_mass=batch.mass, workspace=batch.workspace,
+                                                 device_status=batch.status)
+    torch.cuda.synchronize()
+    masses = rk.split_block_mass(plan, mass)
+    npg = int(w.tables.seg_block_off[1])
+    scores = sum(m[:, :npg].astype(np.float64).sum(axis=0) for m in masses)
+    holed = workloads.punch_holes(w, 0, workloads.lowest_mass_pages(scores, 0.2))
+    batch.w = holed
+    batch.tables = holed.tables
+
+
+def sweep_configs(rk, dev, flush, peak_gbs, skip, cached):
+    """Attention-only time of every config (plan prebuilt, cold L2), as context for the headline workload."""
+    import torch
+    res = {}
+    for name in WORKLOAD_LABEL:
+        if name == skip:
+            a = cached[1]["attention_only"]
+            res[name] = {"unique_kv_bytes": cached[1]["config"]["unique_kv_bytes"], "ms_median": a["ms_median"],
+                         "tbps_unique_kv": a["tbps_unique_kv"], "pct_of_8tbps": a["pct_of_8tbps"]}
+            continue
+        w = load_workload(name)
+        b = DeviceBatch(w, dev)
+        if name == "long_context":
+            punch_long_context(rk, b)
+        plan, _ = run_step(rk, b)
+        torch.cuda.synchronize()
+        kv, _ = algorithmic_bytes(plan, b.w.layout)
+        att = attention_only_times(rk, b, plan, 20, flush)
+        med = statistics.median(att)
+        res[name] = {"unique_kv_bytes": kv, "ms_median": med, "ms_min": min(att),
+                     "tbps_unique_kv": kv / (med * 1e-3) / 1e12,
+                     "pct_of_8tbps": 100.0 * kv / (med * 1e-3) / 1e12 / NOMINAL_HBM_TBPS,
+                     "branch_steps_per_s": b.w.num_branches / (med * 1e-3), "work_items": plan.num_work_items}
+        del b
+        torch.cuda.empty_cache()
+    return res
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -176,6 +176,19 @@ RKSC_API int32_t rksc_branch_decode_attention(const rksc_plan* plan, const void*
                                      void* workspace, size_t workspace_bytes,
                                      int32_t* device_status, void* stream);
 
+/* The same call restricted to some of its launches, so that a profiler or a benchmark can put
+ * CUDA events between them: RKSC_PHASE_SEGMENTS runs the segment-attention kernel (partials and
+ * log2 masses), RKSC_PHASE_MERGE the merge kernel (out and final masses).  The merge phase must
+ * follow the segment phase on the same stream with the same arguments.
+ * rksc_branch_decode_attention == phases (RKSC_PHASE_SEGMENTS | RKSC_PHASE_MERGE). */
+#define RKSC_PHASE_SEGMENTS 1
+#define RKSC_PHASE_MERGE    2
+RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan* plan, const void* q,
+                                     const void* k_pool, const void* v_pool,
+                                     float* out, float* block_mass,
+                                     void* workspace, size_t workspace_bytes,
+                                     int32_t* device_status, void* stream, int32_t phases);
+
 #ifdef __cplusplus
 }
 #endif

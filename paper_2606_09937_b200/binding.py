@@ -26,6 +26,7 @@ EXPORTED_SYMBOLS = (
     "rksc_plan_get_item",
     "rksc_plan_destroy",
     "rksc_branch_decode_attention",
+    "rksc_branch_decode_attention_phases",
 )
 
 
@@ -88,6 +89,8 @@ def lib() -> C.CDLL:
     L.rksc_plan_destroy.argtypes = [C.c_void_p]
     L.rksc_branch_decode_attention.restype = C.c_int32
     L.rksc_branch_decode_attention.argtypes = [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p, C.c_void_p]
+    L.rksc_branch_decode_attention_phases.restype = C.c_int32
+    L.rksc_branch_decode_attention_phases.argtypes = [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p, C.c_void_p, C.c_int32]
     _lib = L
     return L
 
@@ -249,8 +252,11 @@ def rksc_asks_gate(h_branch, h_root, cand_prefix, alpha: float, tau: float,
 
 
 def rksc_branch_decode_attention(plan: Plan, q, k_pool, v_pool, out=None, block_mass=None,
-                                 workspace=None, device_status=None, stream=None, want_mass=True):
-    """Launches the attention.  Returns (out fp32 [B][Hq][d], block_mass fp32 flat or None, device_status)."""
+                                 workspace=None, device_status=None, stream=None, want_mass=True, phases=3):
+    """Launches the attention.  Returns (out fp32 [B][Hq][d], block_mass fp32 flat or None, device_status).
+
+    ``phases`` other than 3 goes through rksc_branch_decode_attention_phases (1 = segment kernel
+    only, 2 = merge only), which exists so that events can be recorded between the launches."""
     import torch
     lay = plan.layout.c
     B = plan.num_branches
@@ -268,11 +274,14 @@ def rksc_branch_decode_attention(plan: Plan, q, k_pool, v_pool, out=None, block_
         workspace = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device=dev)
     if device_status is None:
         device_status = torch.zeros(1, dtype=torch.int32, device=dev)
-    st = lib().rksc_branch_decode_attention(
-        plan._h, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), out.data_ptr(),
-        block_mass.data_ptr() if block_mass is not None else None,
-        workspace.data_ptr(), workspace.numel() * workspace.element_size(),
-        device_status.data_ptr(), _stream_ptr(stream))
+    args = (plan._h, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), out.data_ptr(),
+            block_mass.data_ptr() if block_mass is not None else None,
+            workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+            device_status.data_ptr(), _stream_ptr(stream))
+    if phases == 3:
+        st = lib().rksc_branch_decode_attention(*args)
+    else:
+        st = lib().rksc_branch_decode_attention_phases(*args, int(phases))
     _check(st, "rksc_branch_decode_attention")
     return out, block_mass, device_status
 

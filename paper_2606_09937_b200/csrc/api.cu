@@ -89,8 +89,10 @@ size_t bytes_of(const std::vector<T>& v) {
 
 int32_t upload_plan(rksc_plan* p) {
     HostPlan& H = p->host;
-    const size_t sizes[7] = {bytes_of(H.items),     bytes_of(H.seg_blocks), bytes_of(H.sharers), bytes_of(H.merge_off),
-                             bytes_of(H.merge_rows), bytes_of(H.mass_off),   bytes_of(H.br_nblk)};
+    constexpr int kN = 9;
+    const size_t sizes[kN] = {bytes_of(H.items),      bytes_of(H.seg_blocks), bytes_of(H.sharers),
+                              bytes_of(H.merge_off),  bytes_of(H.merge_rows), bytes_of(H.mass_off),
+                              bytes_of(H.br_nblk),    bytes_of(H.cta_item_off), bytes_of(H.cta_items)};
     size_t total = 0;
     for (size_t s : sizes) total += s;
     if (total == 0) total = 256;
@@ -100,13 +102,14 @@ int32_t upload_plan(rksc_plan* p) {
     } catch (const std::bad_alloc&) {
         return RKSC_ERR_NOMEM;
     }
-    const void* srcs[7] = {H.items.data(),      H.seg_blocks.data(), H.sharers.data(), H.merge_off.data(),
-                           H.merge_rows.data(), H.mass_off.data(),   H.br_nblk.data()};
-    const size_t raw[7] = {H.items.size() * sizeof(WorkItem),   H.seg_blocks.size() * 4, H.sharers.size() * sizeof(Sharer),
-                           H.merge_off.size() * 4,              H.merge_rows.size() * 4, H.mass_off.size() * 8,
-                           H.br_nblk.size() * 4};
-    size_t offs[7], off = 0;
-    for (int i = 0; i < 7; ++i) {
+    const void* srcs[kN] = {H.items.data(),      H.seg_blocks.data(), H.sharers.data(),      H.merge_off.data(),
+                            H.merge_rows.data(), H.mass_off.data(),   H.br_nblk.data(),      H.cta_item_off.data(),
+                            H.cta_items.data()};
+    const size_t raw[kN] = {H.items.size() * sizeof(WorkItem), H.seg_blocks.size() * 4, H.sharers.size() * sizeof(Sharer),
+                            H.merge_off.size() * 4,            H.merge_rows.size() * 4, H.mass_off.size() * 8,
+                            H.br_nblk.size() * 4,              H.cta_item_off.size() * 4, H.cta_items.size() * 4};
+    size_t offs[kN], off = 0;
+    for (int i = 0; i < kN; ++i) {
         offs[i] = off;
         if (raw[i]) std::memcpy(stage.data() + off, srcs[i], raw[i]);
         off += sizes[i];
@@ -130,6 +133,8 @@ int32_t upload_plan(rksc_plan* p) {
     p->dev.merge_rows = reinterpret_cast<const int32_t*>(base + offs[4]);
     p->dev.mass_off = reinterpret_cast<const int64_t*>(base + offs[5]);
     p->dev.br_nblk = reinterpret_cast<const int32_t*>(base + offs[6]);
+    p->dev.cta_item_off = reinterpret_cast<const int32_t*>(base + offs[7]);
+    p->dev.cta_items = reinterpret_cast<const int32_t*>(base + offs[8]);
     p->on_device = true;
     return RKSC_OK;
 }
@@ -249,7 +254,16 @@ extern "C" RKSC_API void rksc_plan_destroy(rksc_plan* plan) {
 extern "C" RKSC_API int32_t rksc_branch_decode_attention(const rksc_plan* plan, const void* q, const void* k_pool,
                                                 const void* v_pool, float* out, float* block_mass, void* workspace,
                                                 size_t workspace_bytes, int32_t* device_status, void* stream) {
+    return rksc_branch_decode_attention_phases(plan, q, k_pool, v_pool, out, block_mass, workspace, workspace_bytes,
+                                               device_status, stream, RKSC_PHASE_SEGMENTS | RKSC_PHASE_MERGE);
+}
+
+extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan* plan, const void* q,
+                                                const void* k_pool, const void* v_pool, float* out,
+                                                float* block_mass, void* workspace, size_t workspace_bytes,
+                                                int32_t* device_status, void* stream, int32_t phases) {
     if (!plan) return RKSC_ERR_INVALID_ARG;
+    if ((phases & ~(RKSC_PHASE_SEGMENTS | RKSC_PHASE_MERGE)) || phases == 0) return RKSC_ERR_INVALID_ARG;
     const HostPlan& H = plan->host;
     if (H.B == 0) return RKSC_OK;
     if (!q || !k_pool || !v_pool || !out) return RKSC_ERR_INVALID_ARG;
@@ -279,6 +293,7 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention(const rksc_plan* plan, 
     a.out = out;
     a.status = device_status;
     a.num_items = (int)H.items.size();
+    a.grid = H.grid;
     a.B = H.B;
     a.Hq = H.layout.num_q_heads;
     a.Hkv = H.layout.num_kv_heads;
@@ -288,8 +303,9 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention(const rksc_plan* plan, 
     a.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_seg_attn_warp(tm_k, tm_v, a, s);
-    if (e == cudaSuccess) e = launch_merge(a, s);
+    cudaError_t e = cudaSuccess;
+    if (phases & RKSC_PHASE_SEGMENTS) e = launch_seg_attn_warp(tm_k, tm_v, a, s);
+    if (e == cudaSuccess && (phases & RKSC_PHASE_MERGE)) e = launch_merge(a, s);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return RKSC_ERR_CUDA;

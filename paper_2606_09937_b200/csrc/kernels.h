@@ -21,6 +21,7 @@ struct AttnArgs {
     float* out;             // [B][Hq][d]
     int32_t* status;        // may be null
     int num_items;
+    int grid;               // persistent CTAs of the segment kernel
     int B, Hq, Hkv, G, head_dim;
     float scale_log2;       // sm_scale * log2(e)
 };

@@ -5,6 +5,8 @@
 #include <cstring>
 #include <new>
 #include <numeric>
+#include <queue>
+#include <utility>
 
 #include "rksc_internal.h"
 
@@ -13,6 +15,12 @@ namespace rksc {
 namespace {
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Relative cost of a work item for packing: streaming its pages plus a fixed start-up share.
+inline int64_t item_cost(const WorkItem& it, int G) {
+    const int nrt = ceil_div(it.num_sharers * G, 16);
+    return (int64_t)it.num_pages * (8 + (nrt - 1)) + 64;
+}
 
 bool csr_ok(const int32_t* off, int n) {
     if (off[0] != 0) return false;
@@ -99,8 +107,9 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
         }
     }
 
-    // chunking: sharer blocks of at most kMaxRowsPerItem rows, KV chunks sized so that the
-    // launch fills the device while partial results stay a few percent of the KV bytes read
+    // chunking: sharer blocks of at most kMaxRowsPerItem rows; KV chunks long enough that the
+    // partial results stay a few percent of the KV bytes read (their size grows with the stacked
+    // rows) and short enough that the persistent CTAs can be packed evenly
     const int per_block = std::max(1, kMaxRowsPerItem / G);
     int64_t total_units = 0;  // page-heads over all (segment, sharer block)
     for (int s = 0; s < S; ++s) {
@@ -110,9 +119,11 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
         P.unique_kv_tokens += P.seg_num_tokens[s];
         total_units += (int64_t)np * L.num_kv_heads * ceil_div(ns, per_block);
     }
-    const int slots = std::max(1, num_sms) * 2;
+    const int max_grid = std::max(1, num_sms) * kCtasPerSm;
     const int kMinChunk = 8;
-    const int upper = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, total_units / slots));
+    const int64_t fair = total_units / max_grid;                     // page-heads per CTA
+    const int cap = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, fair * 2 / 3));
+    const int base = (int)std::min<int64_t>(128, std::max<int64_t>(kMinChunk, fair / 6));
 
     int64_t rows_total = 0;
     for (int s = 0; s < S; ++s) {
@@ -124,7 +135,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
             // balanced split of the sharers
             const int sh_lo = (int)((int64_t)ns * sb / nsb), sh_hi = (int)((int64_t)ns * (sb + 1) / nsb);
             const int rows = (sh_hi - sh_lo) * G;
-            const int want = std::min(upper, std::max(kMinChunk, 2 * rows));
+            const int want = std::min(cap, std::max(base, 2 * rows));
             const int nch = ceil_div(np, want);
             for (int c = 0; c < nch; ++c) {
                 const int p_lo = (int)((int64_t)np * c / nch), p_hi = (int)((int64_t)np * (c + 1) / nch);
@@ -152,9 +163,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
 
     // longest first, so the hardware block scheduler packs the tail with short items
     std::stable_sort(P.items.begin(), P.items.end(), [G](const WorkItem& a, const WorkItem& b) {
-        const int64_t ca = (int64_t)a.num_pages * (3 + ceil_div(a.num_sharers * G, 16));
-        const int64_t cb = (int64_t)b.num_pages * (3 + ceil_div(b.num_sharers * G, 16));
-        return ca > cb;
+        return item_cost(a, G) > item_cost(b, G);
     });
     int32_t row = 0;
     for (auto& it : P.items) {
@@ -162,6 +171,29 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
         row += it.num_sharers * G;
     }
     P.num_partial_rows = row;
+
+    // pack the items onto the persistent CTAs: longest first onto the least loaded CTA
+    {
+        const int n = (int)P.items.size();
+        P.grid = std::min(max_grid, n);
+        std::vector<std::vector<int32_t>> lists(P.grid);
+        using Load = std::pair<int64_t, int>;
+        std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+        for (int c = 0; c < P.grid; ++c) heap.push({0, c});
+        for (int i = 0; i < n; ++i) {
+            Load top = heap.top();
+            heap.pop();
+            lists[top.second].push_back(i);
+            top.first += item_cost(P.items[i], G);
+            heap.push(top);
+        }
+        P.cta_item_off.assign(P.grid + 1, 0);
+        P.cta_items.clear();
+        for (int c = 0; c < P.grid; ++c) {
+            for (int i : lists[c]) P.cta_items.push_back(i);
+            P.cta_item_off[c + 1] = (int32_t)P.cta_items.size();
+        }
+    }
 
     // merge lists: for every (branch, kv head) the partial rows (of head-in-group 0) to combine
     const int nkeys = B * L.num_kv_heads;

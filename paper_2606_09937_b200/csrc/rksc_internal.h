@@ -12,8 +12,11 @@ namespace rksc {
 constexpr int kBlock = RKSC_BLOCK_SIZE;     // tokens per KV page
 constexpr int kMaxRowsPerItem = 64;         // stacked query rows one warp-MMA work item handles
 constexpr int kMaxPagesPerItem = 512;       // page ids a CTA caches in shared memory
-constexpr int kWarpKernelThreads = 128;
-constexpr int kWarpKernelSlots = 12;        // (K page + V page) ring slots per CTA
+constexpr int kConsumerWarps = 4;           // MMA warps of the segment kernel
+constexpr int kWarpKernelThreads = (kConsumerWarps + 1) * 32;   // + one TMA producer warp
+constexpr int kSubPages = 4;                // pages staged per ring slot
+constexpr int kRingSlots = 3;               // ring slots per CTA
+constexpr int kCtasPerSm = 2;               // persistent CTAs per SM
 
 // One CTA's work: a chunk of one segment's pages for one KV head and a block of the
 // segment's sharers.  Stacked rows = num_sharers * G, row r <-> (sharer r / G, head r % G).
@@ -29,6 +32,7 @@ struct WorkItem {
     int32_t seg_page_begin;  // index of the first page within its segment
     int32_t klass;           // 0: warp-MMA kernel
 };
+static_assert(sizeof(WorkItem) == 40, "WorkItem is read as 10 int32");
 
 // A (segment, branch) incidence: where the branch's masses of this segment start.
 struct Sharer {
@@ -39,6 +43,8 @@ struct Sharer {
 
 struct DevicePlan {
     const WorkItem* items = nullptr;
+    const int32_t* cta_item_off = nullptr;  // [grid + 1]
+    const int32_t* cta_items = nullptr;     // item indices, per persistent CTA
     const int32_t* seg_blocks = nullptr;
     const Sharer* sharers = nullptr;
     const int32_t* merge_off = nullptr;   // [B*Hkv + 1]
@@ -50,10 +56,13 @@ struct DevicePlan {
 struct HostPlan {
     rksc_layout layout{};
     int32_t B = 0, S = 0, G = 1;
-    std::vector<int32_t> seg_blocks;      // flattened page ids of the segments that have sharers... all segments
+    std::vector<int32_t> seg_blocks;      // flattened page ids of all segments
     std::vector<int32_t> seg_block_off;
     std::vector<int32_t> seg_num_tokens;
     std::vector<WorkItem> items;
+    int32_t grid = 0;                     // persistent CTAs of the segment kernel
+    std::vector<int32_t> cta_item_off;    // [grid + 1]
+    std::vector<int32_t> cta_items;
     std::vector<Sharer> sharers;
     std::vector<int32_t> seg_sharer_off;  // [S+1]
     std::vector<int32_t> merge_off;
