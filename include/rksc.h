@@ -45,6 +45,8 @@ extern "C" {
 #endif
 
 RKSC_API const char* rksc_strerror(int32_t status);
+/* Text of the CUDA error behind the calling thread's most recent RKSC_ERR_CUDA from a launch. */
+RKSC_API const char* rksc_last_cuda_error(void);
 
 /* ------------------------------------------------------------------------------------------
  * ASKS similarity gate  (paper Eq. 2 and Algorithm 2)
@@ -125,8 +127,9 @@ RKSC_API void rksc_tables_free(rksc_tables* t);
  * device's SM count, lays out the partial-result workspace and the block-mass output, and
  * uploads its lists to the current device (synchronously; it may allocate device memory).
  * Without a CUDA device the plan is host-only: it can be queried but not run.
- * A plan is immutable and may be used from several streams at once with distinct
- * workspaces.  It does not keep pointers into `tables`.
+ * A plan holds a small device-side work counter that a launch uses and rewinds, so a plan may
+ * be in flight on one stream at a time (create one plan per concurrent stream).  It does not
+ * keep pointers into `tables`.
  * ------------------------------------------------------------------------------------------ */
 typedef struct rksc_plan rksc_plan;
 

@@ -18,6 +18,7 @@ _lib = None
 
 EXPORTED_SYMBOLS = (
     "rksc_strerror",
+    "rksc_last_cuda_error",
     "rksc_asks_gate",
     "rksc_tables_from_gate",
     "rksc_tables_free",
@@ -33,7 +34,10 @@ EXPORTED_SYMBOLS = (
 class RkscError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = int(status)
-        super().__init__(f"{where}: {rksc_strerror(status)} (status {status})")
+        detail = ""
+        if status == -5:
+            detail = " [" + lib().rksc_last_cuda_error().decode() + "]"
+        super().__init__(f"{where}: {rksc_strerror(status)} (status {status}){detail}")
 
 
 class _CLayout(C.Structure):
@@ -72,6 +76,8 @@ def lib() -> C.CDLL:
     i32p = C.POINTER(C.c_int32)
     L.rksc_strerror.restype = C.c_char_p
     L.rksc_strerror.argtypes = [C.c_int32]
+    L.rksc_last_cuda_error.restype = C.c_char_p
+    L.rksc_last_cuda_error.argtypes = []
     L.rksc_asks_gate.restype = C.c_int32
     L.rksc_asks_gate.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                  C.c_int32, C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]

@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 REPO_DIR = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "librksc.so")
-SOURCES = ["api.cu", "plan.cpp", "gate.cu", "attn_warp.cu", "merge.cu"]
+SOURCES = ["api.cu", "plan.cpp", "gate.cu", "attn_warp.cu", "attn_tc.cu", "merge.cu"]
 HEADERS = ["rksc_internal.h", "kernels.h"]
 
 
@@ -31,9 +31,11 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every CUDA source for sm_100a and link the shared library; returns its path."""
-    if not force and not _stale():
+def build(force: bool = False, verbose: bool = False, extra_flags=(), out_path: str = LIB_PATH) -> str:
+    """Compile every CUDA source for sm_100a and link the shared library; returns its path.
+
+    ``extra_flags`` / ``out_path`` build a variant (e.g. ``-DRKSC_WAIT_PROFILE``) beside the product library."""
+    if out_path == LIB_PATH and not force and not _stale():
         return LIB_PATH
     cmd = [
         _nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -43,15 +45,16 @@ def build(force: bool = False, verbose: bool = False) -> str:
     ]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += list(extra_flags)
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
-    cmd += ["-o", LIB_PATH + ".tmp"]
+    cmd += ["-o", out_path + ".tmp"]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-    os.replace(LIB_PATH + ".tmp", LIB_PATH)
+    os.replace(out_path + ".tmp", out_path)
     if verbose:
         print(res.stderr)
-    return LIB_PATH
+    return out_path
 
 
 if __name__ == "__main__":

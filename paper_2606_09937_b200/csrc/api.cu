@@ -18,6 +18,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 std::mutex g_mu;
+thread_local cudaError_t g_last_cuda = cudaSuccess;   // the CUDA error behind the last RKSC_ERR_CUDA of this thread
+
 EncodeTiledFn g_encode = nullptr;
 constexpr int kMaxDevices = 64;
 int g_dev_state[kMaxDevices];   // 0 unknown, 1 ready (sm_100 family, kernels configured), -1 unsupported, -2 cuda error
@@ -89,10 +91,10 @@ size_t bytes_of(const std::vector<T>& v) {
 
 int32_t upload_plan(rksc_plan* p) {
     HostPlan& H = p->host;
-    constexpr int kN = 9;
+    constexpr int kN = 8;
     const size_t sizes[kN] = {bytes_of(H.items),      bytes_of(H.seg_blocks), bytes_of(H.sharers),
                               bytes_of(H.merge_off),  bytes_of(H.merge_rows), bytes_of(H.mass_off),
-                              bytes_of(H.br_nblk),    bytes_of(H.cta_item_off), bytes_of(H.cta_items)};
+                              bytes_of(H.br_nblk),    256 /* counters, zeroed */};
     size_t total = 0;
     for (size_t s : sizes) total += s;
     if (total == 0) total = 256;
@@ -103,11 +105,10 @@ int32_t upload_plan(rksc_plan* p) {
         return RKSC_ERR_NOMEM;
     }
     const void* srcs[kN] = {H.items.data(),      H.seg_blocks.data(), H.sharers.data(),      H.merge_off.data(),
-                            H.merge_rows.data(), H.mass_off.data(),   H.br_nblk.data(),      H.cta_item_off.data(),
-                            H.cta_items.data()};
+                            H.merge_rows.data(), H.mass_off.data(),   H.br_nblk.data(),      nullptr};
     const size_t raw[kN] = {H.items.size() * sizeof(WorkItem), H.seg_blocks.size() * 4, H.sharers.size() * sizeof(Sharer),
                             H.merge_off.size() * 4,            H.merge_rows.size() * 4, H.mass_off.size() * 8,
-                            H.br_nblk.size() * 4,              H.cta_item_off.size() * 4, H.cta_items.size() * 4};
+                            H.br_nblk.size() * 4,              0};
     size_t offs[kN], off = 0;
     for (int i = 0; i < kN; ++i) {
         offs[i] = off;
@@ -133,8 +134,7 @@ int32_t upload_plan(rksc_plan* p) {
     p->dev.merge_rows = reinterpret_cast<const int32_t*>(base + offs[4]);
     p->dev.mass_off = reinterpret_cast<const int64_t*>(base + offs[5]);
     p->dev.br_nblk = reinterpret_cast<const int32_t*>(base + offs[6]);
-    p->dev.cta_item_off = reinterpret_cast<const int32_t*>(base + offs[7]);
-    p->dev.cta_items = reinterpret_cast<const int32_t*>(base + offs[8]);
+    p->dev.counters = reinterpret_cast<int32_t*>(base + offs[7]);
     p->on_device = true;
     return RKSC_OK;
 }
@@ -168,11 +168,14 @@ extern "C" RKSC_API int32_t rksc_asks_gate(const float* h_branch, const float* h
     cudaError_t e = launch_asks_gate(h_branch, h_root, cand_prefix, B, P, L, D, alpha, tau, branch_to_prefix, sigma,
                                      static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {
+        g_last_cuda = e;
         cudaGetLastError();
         return RKSC_ERR_CUDA;
     }
     return RKSC_OK;
 }
+
+extern "C" RKSC_API const char* rksc_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda); }
 
 extern "C" RKSC_API int32_t rksc_plan_create(const rksc_layout* layout, const rksc_tables* tables, rksc_plan** out) {
     if (!layout || !tables || !out) return RKSC_ERR_INVALID_ARG;
@@ -292,8 +295,11 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
     a.block_mass = block_mass;
     a.out = out;
     a.status = device_status;
+    a.counters = plan->dev.counters;
     a.num_items = (int)H.items.size();
-    a.grid = H.grid;
+    a.num_tc_items = H.num_tc_items;
+    a.grid_warp = H.grid_warp;
+    a.grid_tc = H.grid_tc;
     a.B = H.B;
     a.Hq = H.layout.num_q_heads;
     a.Hkv = H.layout.num_kv_heads;
@@ -304,9 +310,13 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaSuccess;
-    if (phases & RKSC_PHASE_SEGMENTS) e = launch_seg_attn_warp(tm_k, tm_v, a, s);
+    if (phases & RKSC_PHASE_SEGMENTS) {
+        e = launch_seg_attn_tc(tm_k, tm_v, a, s);
+        if (e == cudaSuccess) e = launch_seg_attn_warp(tm_k, tm_v, a, s, /*after_tc=*/a.grid_tc > 0);
+    }
     if (e == cudaSuccess && (phases & RKSC_PHASE_MERGE)) e = launch_merge(a, s);
     if (e != cudaSuccess) {
+        g_last_cuda = e;
         cudaGetLastError();
         return RKSC_ERR_CUDA;
     }

@@ -20,8 +20,10 @@ struct AttnArgs {
     float* block_mass;      // may be null; holds log2 masses between the two launches
     float* out;             // [B][Hq][d]
     int32_t* status;        // may be null
+    int32_t* counters;      // [2]: next work item, CTAs done; zero between launches
     int num_items;
-    int grid;               // persistent CTAs of the segment kernel
+    int num_tc_items;       // items [0, num_tc_items) go to the tcgen05 kernel, the rest to the warp kernel
+    int grid_warp, grid_tc; // persistent CTAs of the two segment kernels
     int B, Hq, Hkv, G, head_dim;
     float scale_log2;       // sm_scale * log2(e)
 };
@@ -30,8 +32,14 @@ struct AttnArgs {
 cudaError_t configure_attention_kernels();
 size_t warp_kernel_smem_bytes(int head_dim);
 
+size_t tc_kernel_smem_bytes();
+
+// after_tc: the tcgen05 kernel was launched just before on the same stream; the warp kernel then
+// starts as that one drains (programmatic dependent launch) and waits for it before it exits.
 cudaError_t launch_seg_attn_warp(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnArgs& a,
-                                 cudaStream_t stream);
+                                 cudaStream_t stream, bool after_tc);
+cudaError_t launch_seg_attn_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnArgs& a,
+                               cudaStream_t stream);
 cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream);
 
 }  // namespace rksc

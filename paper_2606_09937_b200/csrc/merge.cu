@@ -1,19 +1,25 @@
 // Log-sum-exp merge of the partial results of one (branch, query head), and the final
 // normalisation of the per-block softmax masses.
 //
-// The segment kernels leave, for every (segment chunk, row), a normalised partial output and its
+// The segment kernel leaves, for every (segment chunk, row), a normalised partial output and its
 // log2-sum-exp, and in block_mass the log2 of every page's unnormalised mass.  Here:
 //   LSE  = log2 sum_p 2^lse_p
 //   out  = sum_p 2^(lse_p - LSE) * O_p
 //   mass_j = 2^(logmass_j - LSE)
 // which is exactly softmax attention over the concatenation of the branch's segments.
+//
+// One warp per (branch, head): lanes split the head dimension four columns each (16-byte loads of
+// the partial rows) and stride over the parts and the blocks.  The kernel is launched with
+// programmatic stream serialisation: its blocks may become resident while the segment kernel
+// drains, read their (plan-owned) part lists, and then wait for the segment kernel's results.
 #include "kernels.h"
 
 namespace rksc {
 
 namespace {
 
-constexpr int kMergeThreads = 128;
+constexpr int kMergeWarps = 8;
+constexpr int kMergeThreads = kMergeWarps * 32;
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -23,51 +29,68 @@ __device__ __forceinline__ float fast_exp2(float x) {
 
 __global__ void __launch_bounds__(kMergeThreads)
 merge_kernel(const AttnArgs a) {
-    const int bh = blockIdx.x;
-    const int b = bh / a.Hq, h = bh % a.Hq;
-    const int kvh = h / a.G, gi = h % a.G;
+    const int lane = threadIdx.x & 31;
+    const int bh = blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
+    const bool live = bh < a.B * a.Hq;
+    int b = 0, h = 0, lo = 0, hi = 0;
+    if (live) {
+        b = bh / a.Hq;
+        h = bh % a.Hq;
+        const int key = b * a.Hkv + h / a.G;
+        lo = a.plan.merge_off[key];
+        hi = a.plan.merge_off[key + 1];
+    }
+    const int gi = h % a.G;
     const int HD = a.head_dim;
-    const int lo = a.plan.merge_off[b * a.Hkv + kvh], hi = a.plan.merge_off[b * a.Hkv + kvh + 1];
-    const int tid = threadIdx.x;
-    __shared__ float red[kMergeThreads / 32];
-    __shared__ float s_lse;
+    // the first 32 part rows of this warp's list (plan data: readable before the dependency resolves)
+    int row_l = (lo + lane < hi) ? a.plan.merge_rows[lo + lane] + gi : -1;
 
-    // max and sum of the parts' log2-sum-exp (block reduction; the list is short)
+    // everything below reads what the segment kernel wrote
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!live) return;
+
+    // LSE over the parts
     float mx = -INFINITY;
-    for (int i = lo + tid; i < hi; i += kMergeThreads) mx = fmaxf(mx, a.part_lse[a.plan.merge_rows[i] + gi]);
+    for (int i = lo + lane; i < hi; i += 32) {
+        const int row = (i < lo + 32) ? row_l : a.plan.merge_rows[i] + gi;
+        mx = fmaxf(mx, a.part_lse[row]);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if ((tid & 31) == 0) red[tid >> 5] = mx;
-    __syncthreads();
-    mx = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
-    __syncthreads();
     float sum = 0.f;
-    for (int i = lo + tid; i < hi; i += kMergeThreads) sum += fast_exp2(a.part_lse[a.plan.merge_rows[i] + gi] - mx);
+    for (int i = lo + lane; i < hi; i += 32) {
+        const int row = (i < lo + 32) ? row_l : a.plan.merge_rows[i] + gi;
+        sum += fast_exp2(a.part_lse[row] - mx);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if ((tid & 31) == 0) red[tid >> 5] = sum;
-    __syncthreads();
-    if (tid == 0) s_lse = mx + log2f((red[0] + red[1]) + (red[2] + red[3]));
-    __syncthreads();
-    const float lse = s_lse;
+    const float lse = mx + log2f(sum);
 
-    float* out = a.out + (size_t)bh * HD;
-    if (hi == lo) {   // the branch attends to nothing
-        for (int c = tid; c < HD; c += kMergeThreads) out[c] = 0.f;
-        return;
-    }
-    for (int c = tid; c < HD; c += kMergeThreads) {
-        float acc = 0.f;
-        for (int i = lo; i < hi; ++i) {
-            const int row = a.plan.merge_rows[i] + gi;
-            acc += fast_exp2(a.part_lse[row] - lse) * a.part_o[(size_t)row * HD + c];
+    // out: lane owns columns 4*lane .. 4*lane+3
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const bool has_cols = 4 * lane < HD;
+    for (int i0 = lo; i0 < hi; i0 += 32) {
+        const int n = min(32, hi - i0);
+        const int my_row = (i0 == lo) ? row_l : ((i0 + lane < hi) ? a.plan.merge_rows[i0 + lane] + gi : -1);
+        const float my_w = (my_row >= 0) ? fast_exp2(a.part_lse[my_row] - lse) : 0.f;
+        for (int j = 0; j < n; ++j) {
+            const int row = __shfl_sync(0xffffffffu, my_row, j);
+            const float w = __shfl_sync(0xffffffffu, my_w, j);
+            if (has_cols) {
+                const float4 v = *reinterpret_cast<const float4*>(a.part_o + (size_t)row * HD + 4 * lane);
+                acc.x += w * v.x;
+                acc.y += w * v.y;
+                acc.z += w * v.z;
+                acc.w += w * v.w;
+            }
         }
-        out[c] = acc;
     }
-    if (a.block_mass != nullptr) {
+    if (has_cols) *reinterpret_cast<float4*>(a.out + (size_t)bh * HD + 4 * lane) = acc;   // zeros when there are no parts
+
+    if (a.block_mass != nullptr && hi > lo) {
         const int nblk = a.plan.br_nblk[b];
         float* mass = a.block_mass + a.plan.mass_off[b] * a.Hq + (int64_t)h * nblk;
-        for (int j = tid; j < nblk; j += kMergeThreads) mass[j] = fast_exp2(mass[j] - lse);
+        for (int j = lane; j < nblk; j += 32) mass[j] = fast_exp2(mass[j] - lse);
     }
 }
 
@@ -76,8 +99,17 @@ merge_kernel(const AttnArgs a) {
 cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream) {
     const int n = a.B * a.Hq;
     if (n == 0) return cudaSuccess;
-    merge_kernel<<<n, kMergeThreads, 0, stream>>>(a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((n + kMergeWarps - 1) / kMergeWarps, 1, 1);
+    cfg.blockDim = dim3(kMergeThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, merge_kernel, a);
 }
 
 }  // namespace rksc

@@ -5,8 +5,6 @@
 #include <cstring>
 #include <new>
 #include <numeric>
-#include <queue>
-#include <utility>
 
 #include "rksc_internal.h"
 
@@ -20,6 +18,11 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline int64_t item_cost(const WorkItem& it, int G) {
     const int nrt = ceil_div(it.num_sharers * G, 16);
     return (int64_t)it.num_pages * (8 + (nrt - 1)) + 64;
+}
+
+bool env_flag(const char* name) {
+    const char* v = std::getenv(name);
+    return v && v[0] && v[0] != '0';
 }
 
 bool csr_ok(const int32_t* off, int n) {
@@ -37,7 +40,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     if (L.block_size != kBlock) return RKSC_ERR_UNSUPPORTED;
     if (L.head_dim != 64 && L.head_dim != 128) return RKSC_ERR_UNSUPPORTED;
     const int G = L.num_q_heads / L.num_kv_heads;
-    if (G > kMaxRowsPerItem) return RKSC_ERR_UNSUPPORTED;
+    if (G > kMaxRowsPerItem) return RKSC_ERR_UNSUPPORTED;   // one branch's heads of a KV head stay in one item
     if ((int64_t)L.num_pool_blocks * L.num_kv_heads * kBlock >= (int64_t)1 << 31) return RKSC_ERR_UNSUPPORTED;
     if (t.num_branches < 0 || t.num_segments < 0) return RKSC_ERR_INVALID_ARG;
     if (!t.seg_block_off || !t.br_seg_off) return RKSC_ERR_INVALID_ARG;
@@ -107,17 +110,23 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
         }
     }
 
-    // chunking: sharer blocks of at most kMaxRowsPerItem rows; KV chunks long enough that the
-    // partial results stay a few percent of the KV bytes read (their size grows with the stacked
-    // rows) and short enough that the persistent CTAs can be packed evenly
-    const int per_block = std::max(1, kMaxRowsPerItem / G);
+    // Work items.  A segment whose stacked rows (sharers x G) reach kTcMinRows goes to the
+    // tensor-core (tcgen05) kernel in sharer blocks of up to 128 rows; the rest goes to the
+    // warp-MMA kernel in blocks of up to 64 rows.  KV chunks are long enough that the partial
+    // results stay a few percent of the KV bytes read (their size grows with the stacked rows)
+    // and short enough that the persistent CTAs end together.
+    const bool tc_ok = (L.head_dim == 128) && !env_flag("RKSC_DISABLE_TC");
+    auto seg_rows_per_block = [&](int ns) {
+        const bool tc = tc_ok && ns * G >= kTcMinRows;
+        return std::max(1, (tc ? kTcMaxRows : kMaxRowsPerItem) / G);
+    };
     int64_t total_units = 0;  // page-heads over all (segment, sharer block)
     for (int s = 0; s < S; ++s) {
         const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
         const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
         if (ns == 0 || np == 0) continue;
         P.unique_kv_tokens += P.seg_num_tokens[s];
-        total_units += (int64_t)np * L.num_kv_heads * ceil_div(ns, per_block);
+        total_units += (int64_t)np * L.num_kv_heads * ceil_div(ns, seg_rows_per_block(ns));
     }
     const int max_grid = std::max(1, num_sms) * kCtasPerSm;
     const int kMinChunk = 8;
@@ -130,11 +139,12 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
         const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
         const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
         if (ns == 0 || np == 0) continue;
-        const int nsb = ceil_div(ns, per_block);
+        const int nsb = ceil_div(ns, seg_rows_per_block(ns));
         for (int sb = 0; sb < nsb; ++sb) {
             // balanced split of the sharers
             const int sh_lo = (int)((int64_t)ns * sb / nsb), sh_hi = (int)((int64_t)ns * (sb + 1) / nsb);
             const int rows = (sh_hi - sh_lo) * G;
+            const int klass = (tc_ok && rows >= kTcMinRows) ? 1 : 0;
             const int want = std::min(cap, std::max(base, 2 * rows));
             const int nch = ceil_div(np, want);
             for (int c = 0; c < nch; ++c) {
@@ -152,7 +162,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
                     it.num_sharers = sh_hi - sh_lo;
                     it.part_row_base = 0;  // set after sorting
                     it.seg_page_begin = p_lo;
-                    it.klass = 0;
+                    it.klass = klass;
                     P.items.push_back(it);
                     rows_total += rows;
                 }
@@ -161,39 +171,22 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     }
     if (rows_total >= ((int64_t)1 << 31)) return RKSC_ERR_UNSUPPORTED;
 
-    // longest first, so the hardware block scheduler packs the tail with short items
+    // tensor-core items first, then warp-MMA items; within a class longest first, so that the
+    // CTAs, which claim items in this order, finish together
     std::stable_sort(P.items.begin(), P.items.end(), [G](const WorkItem& a, const WorkItem& b) {
+        if (a.klass != b.klass) return a.klass > b.klass;
         return item_cost(a, G) > item_cost(b, G);
     });
     int32_t row = 0;
+    P.num_tc_items = 0;
     for (auto& it : P.items) {
         it.part_row_base = row;
         row += it.num_sharers * G;
+        P.num_tc_items += it.klass;
     }
     P.num_partial_rows = row;
-
-    // pack the items onto the persistent CTAs: longest first onto the least loaded CTA
-    {
-        const int n = (int)P.items.size();
-        P.grid = std::min(max_grid, n);
-        std::vector<std::vector<int32_t>> lists(P.grid);
-        using Load = std::pair<int64_t, int>;
-        std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-        for (int c = 0; c < P.grid; ++c) heap.push({0, c});
-        for (int i = 0; i < n; ++i) {
-            Load top = heap.top();
-            heap.pop();
-            lists[top.second].push_back(i);
-            top.first += item_cost(P.items[i], G);
-            heap.push(top);
-        }
-        P.cta_item_off.assign(P.grid + 1, 0);
-        P.cta_items.clear();
-        for (int c = 0; c < P.grid; ++c) {
-            for (int i : lists[c]) P.cta_items.push_back(i);
-            P.cta_item_off[c + 1] = (int32_t)P.cta_items.size();
-        }
-    }
+    P.grid_tc = std::min(std::max(1, num_sms), P.num_tc_items);
+    P.grid_warp = std::min(max_grid, (int)P.items.size() - P.num_tc_items);
 
     // merge lists: for every (branch, kv head) the partial rows (of head-in-group 0) to combine
     const int nkeys = B * L.num_kv_heads;
