@@ -6,19 +6,20 @@
 // branch (the shared-prefix read that replaces the paper's per-branch copies of the prefix cache,
 // Algorithm 1 line 3 / Section 2.2).  Here the product really is a dense contraction:
 //   S[128 x 64]  = Q[128 x d] K^T        (tcgen05.mma, A and B K-major in 128-byte-swizzled smem)
-//   O[128 x d]  += P[128 x 64] V         (A = P written to smem by the softmax warps, B = V MN-major)
-// with both accumulators in tensor memory.  One persistent CTA per SM, ten warps:
+//   O[128 x d]  += P[128 x 64] V         (A = P read from tensor memory, B = V MN-major in smem)
+// with S, P and O in tensor memory.  One persistent CTA per SM, eleven warps:
 //   warps 0-3 / 4-7  two softmax warpgroups; thread = one stacked row (TMEM lane).  They take
 //                    alternate 64-token slots of an item, each with its own S and O accumulator and
 //                    its own running (max, sum), merged at the end of the item.  Per slot: tcgen05.ld
 //                    of the S row, scale + mask + online softmax in base 2, per-page softmax mass
-//                    (log2, absolute) to global memory, P as bf16 to shared memory; O is rescaled in
-//                    TMEM (tcgen05.ld / st) only when some running maximum of the warp moved.
+//                    (log2, absolute) to global memory, P as bf16 back to tensor memory (tcgen05.st);
+//                    O is rescaled in TMEM (tcgen05.ld / st) only when a running maximum of the warp moved.
 //   warp 8           producer: claims work items from a global counter and streams their pages by
-//                    TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a four-slot
+//                    TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a five-slot
 //                    ring, four pages per slot, with a header per slot that the other warps follow.
-//   warp 9           allocates TMEM; one lane issues the MMAs: S of slot i+1 is issued before P V of
-//                    slot i, so the tensor pipe works while the other warpgroup is in its softmax.
+//   warps 9, 10      MMA issuers, one per warpgroup (one lane each; warp 9 also allocates TMEM): S of the
+//                    warpgroup's next slot is issued before P V of its previous one, so S is waiting when
+//                    the warpgroup comes out of its softmax and the tensor pipe runs under both softmaxes.
 // Completion of MMAs is signalled with tcgen05.commit onto mbarriers (S ready, O ready / P free,
 // ring slot free).  Every wait is bounded: on expiry the CTA records RKSC_ERR_DEVICE_TIMEOUT,
 // stops issuing work, skips further waits, frees its TMEM and returns.
@@ -33,25 +34,23 @@ namespace {
 constexpr int HD = 128;
 constexpr int kSmWarps = 8;                       // softmax warps (two warpgroups)
 constexpr int kProducerWarp = kSmWarps;           // 8
-constexpr int kMmaWarp = kSmWarps + 1;            // 9
-constexpr int kTcThreads = (kSmWarps + 2) * 32;   // 320
-constexpr int kNS = 4;                            // ring slots
+constexpr int kMmaWarp = kSmWarps + 1;            // 9 and 10: MMA issuers of warpgroup 0 and 1
+constexpr int kTcThreads = (kSmWarps + 3) * 32;   // 352
+constexpr int kNS = 5;                            // ring slots
 constexpr int kSlotTokens = 64;                   // 4 pages
 constexpr int kKBytes = kSlotTokens * HD * 2;     // K (or V) of a slot: [half][64 tokens][128 B] = 16 KiB
 constexpr int kSlotBytes = 2 * kKBytes;
-constexpr int kRingBytes = kNS * kSlotBytes;      // 128 KiB
+constexpr int kRingBytes = kNS * kSlotBytes;      // 160 KiB
 constexpr int kQOff = kRingBytes;                 // Q tile [half][128 rows][128 B]
 constexpr int kQBytes = 128 * HD * 2;             // 32 KiB
-constexpr int kPOff = kQOff + kQBytes;            // P tiles, one per warpgroup: [128 rows][128 B]
-constexpr int kPBytes = 128 * 128;                // 16 KiB
-constexpr int kMlOff = kPOff + 2 * kPBytes;       // (m, l) exchange [2][128] float2
+constexpr int kMlOff = kQOff + kQBytes;           // (m, l) exchange [2][128] float2
 constexpr int kBarOff = kMlOff + 2 * 128 * 8;
 // mbarriers
 constexpr int kBarFull = 0;                       // [kNS]  producer -> everyone: slot landed (+ header)
-constexpr int kBarEmpty = kBarFull + kNS;         // [kNS]  slot reusable: P V committed + 8 header readers
+constexpr int kBarEmpty = kBarFull + kNS;         // [kNS]  slot reusable: P V committed + 10 header readers
 constexpr int kBarSFull = kBarEmpty + kNS;        // [2]    S of the warpgroup's slot is in TMEM
 constexpr int kBarSFree = kBarSFull + 2;          // [2]    the warpgroup has copied S to registers
-constexpr int kBarPFull = kBarSFree + 2;          // [2]    P of the slot is in shared memory
+constexpr int kBarPFull = kBarSFree + 2;          // [2]    P of the slot is in tensor memory
 constexpr int kBarODone = kBarPFull + 2;          // [2]    P V of the slot has completed
 constexpr int kBarQFull = kBarODone + 2;          // Q tile of the item is in shared memory
 constexpr int kBarEpiA = kBarQFull + 1;           // item epilogue: (m, l) published
@@ -62,8 +61,9 @@ constexpr int kTmemPtrOff = kHdrOff + kNS * 64;
 constexpr int kFlagOff = kTmemPtrOff + 16;
 constexpr int kSmemTotal = kFlagOff + 16;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;                     // S[wg] at columns 64*wg
-constexpr uint32_t kColO = 128;                   // O[wg] at columns 128 + 128*wg
+constexpr uint32_t kColS = 0;                     // S[wg]: 64 fp32 columns at 64*wg
+constexpr uint32_t kColO = 128;                   // O[wg]: 128 fp32 columns at 128 + 128*wg
+constexpr uint32_t kColP = 384;                   // P[wg]: 64 bf16 = 32 columns at 384 + 32*wg
 
 struct __align__(16) SlotHeader {
     int32_t item;        // index of the work item, -1: no more work
@@ -159,6 +159,17 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// A operand (128 x 16 bf16, two values per 32-bit column) read from tensor memory
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // 32 consecutive columns of this thread's TMEM lane
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -186,6 +197,22 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+#ifdef RKSC_WAIT_PROFILE
+// Development aid: cycles per CTA spent in the waits of the MMA lane ([0..4]: total, slot landed,
+// S buffer free, P ready, Q ready) and of softmax warp 0 ([8..15]: total, slot landed, S ready,
+// previous P V done, epilogue A, epilogue B, slots, items).
+__device__ unsigned long long g_tc_prof[384][16];
+#define TCPROF_DECL unsigned long long tcp[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long tcp_begin = clock64()
+#define TCPROF_WAIT(i, stmt) { const long long _t = clock64(); stmt; tcp[i] += (unsigned long long)(clock64() - _t); }
+#define TCPROF_MARK(i) { const long long _n = clock64(); tcq[i] += (unsigned long long)(_n - tcq_t); tcq_t = _n; }
+#define TCPROF_FLUSH(base) { tcp[0] = (unsigned long long)(clock64() - tcp_begin); for (int _i = 0; _i < 8; ++_i) g_tc_prof[blockIdx.x][base + _i] = tcp[_i]; }
+#else
+#define TCPROF_DECL
+#define TCPROF_WAIT(i, stmt) stmt
+#define TCPROF_MARK(i)
+#define TCPROF_FLUSH(base)
+#endif
+
 __global__ void __launch_bounds__(kTcThreads, 1)
 seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const AttnArgs a) {
@@ -202,7 +229,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (tid == 0) {
         for (int i = 0; i < kNS; ++i) {
             mbar_init(bar(kBarFull + i), 1);
-            mbar_init(bar(kBarEmpty + i), 1 + kSmWarps);
+            mbar_init(bar(kBarEmpty + i), 1 + kSmWarps + 2);   // P V commit, 8 softmax warps, 2 MMA issuers
         }
         for (int w = 0; w < 2; ++w) {
             mbar_init(bar(kBarSFull + w), 1);
@@ -218,7 +245,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         // the kernels that follow on the stream may be made resident early; they wait themselves
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     }
-    if (warp == kMmaWarp) {
+    if (warp == kMmaWarp) {   // one warp allocates (and later frees) the tensor memory
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + kTmemPtrOff),
                      "r"(kTmemCols)
                      : "memory");
@@ -319,68 +346,74 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 __threadfence();
             }
         }
-    } else if (warp == kMmaWarp) {
-        // ------------------------------------ MMA issuer ------------------------------------
+    } else if (warp >= kMmaWarp) {
+        // ------------------------- MMA issuers: warp 9 for warpgroup 0, warp 10 for warpgroup 1 -------------------------
+        // Each walks every slot header (to see item boundaries) and issues the MMAs of its own
+        // warpgroup's slots: S of the next own slot goes out before P V of the previous one, so S
+        // is ready by the time the warpgroup finishes its softmax.
         if (lane == 0) {
             constexpr uint32_t kIdescQK = instr_desc(kSlotTokens, 0);
             constexpr uint32_t kIdescPV = instr_desc(HD, 1);
-            int cw[2] = {0, 0};          // slots issued per warpgroup (all items)
-            bool first_pv[2] = {true, true};
+            const int wg = warp - kMmaWarp;
+            int c = 0;                   // own slots issued (all items)
+            bool first_pv = true;
             int item_k = -1;
-            int pend_slot = -1, pend_wg = 0, pend_npg = 0, pend_c = 0;
+            int pend_slot = -1, pend_npg = 0, pend_c = 0;
+            TCPROF_DECL;
             auto flush_pv = [&]() {
                 if (pend_slot < 0) return;
-                wait_or_abort(bar(kBarPFull + pend_wg), (uint32_t)pend_c & 1u);
+                TCPROF_WAIT(3, wait_or_abort(bar(kBarPFull + wg), (uint32_t)pend_c & 1u));
                 if (!*s_abort) {
                     tc_fence_after();
-                    const uint32_t pbase = sbase + kPOff + pend_wg * kPBytes;
                     const uint32_t vbase = sbase + pend_slot * kSlotBytes + kKBytes;
-                    for (int j = 0; j < pend_npg; ++j) {
-                        const uint64_t ad = smem_desc(pbase + j * 32, 16, 1024);
+                    TCPROF_WAIT(6, for (int j = 0; j < pend_npg; ++j) {
                         const uint64_t bd = smem_desc(vbase + j * 2048, 8192, 1024);
-                        umma(tmem + kColO + pend_wg * 128, ad, bd, kIdescPV, (first_pv[pend_wg] && j == 0) ? 0u : 1u);
-                    }
-                    first_pv[pend_wg] = false;
-                    tc_commit(bar(kBarODone + pend_wg));
-                    tc_commit(bar(kBarEmpty + pend_slot));
+                        umma_ts(tmem + kColO + wg * 128, tmem + kColP + wg * 32 + j * 8, bd, kIdescPV,
+                                (first_pv && j == 0) ? 0u : 1u);
+                    });
+                    first_pv = false;
+                    TCPROF_WAIT(7, tc_commit(bar(kBarODone + wg));
+                    tc_commit(bar(kBarEmpty + pend_slot)));
                 }
                 pend_slot = -1;
             };
             for (int seq = 0; !*s_abort; ++seq) {
                 const int slot = seq % kNS;
-                wait_or_abort(bar(kBarFull + slot), (uint32_t)(seq / kNS) & 1u);
+                TCPROF_WAIT(1, wait_or_abort(bar(kBarFull + slot), (uint32_t)(seq / kNS) & 1u));
                 if (*s_abort) break;
-                const int item = s_hdr[slot].item;
-                if (item < 0) break;
-                const int g = s_hdr[slot].group, npg = s_hdr[slot].num_pages;
-                const int wg = g & 1;
+                const int4 hdr = *reinterpret_cast<const int4*>(&s_hdr[slot]);   // item, group, pages, last
+                if (hdr.x < 0) break;
+                const int g = hdr.y, npg = hdr.z;
+                const bool own = (g & 1) == wg;
+                // a slot of the other warpgroup is only looked at: hand the header back
+                if (!own) mbar_arrive(bar(kBarEmpty + slot));
                 if (g == 0) {
                     flush_pv();
                     ++item_k;
-                    wait_or_abort(bar(kBarQFull), (uint32_t)item_k & 1u);
+                    TCPROF_WAIT(4, wait_or_abort(bar(kBarQFull), (uint32_t)item_k & 1u));
                     if (*s_abort) break;
-                    first_pv[0] = first_pv[1] = true;
+                    first_pv = true;
                 }
-                const int c = cw[wg];
-                if (c > 0) wait_or_abort(bar(kBarSFree + wg), (uint32_t)(c - 1) & 1u);
+                if (!own) continue;
+                if (c > 0) TCPROF_WAIT(2, wait_or_abort(bar(kBarSFree + wg), (uint32_t)(c - 1) & 1u));
                 if (*s_abort) break;
                 tc_fence_after();
                 const uint32_t qbase = sbase + kQOff, kbase = sbase + slot * kSlotBytes;
-#pragma unroll
-                for (int ks = 0; ks < HD / 16; ++ks) {
+                TCPROF_WAIT(5, for (int ks = 0; ks < HD / 16; ++ks) {
                     const uint64_t ad = smem_desc(qbase + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
                     const uint64_t bd = smem_desc(kbase + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
                     umma(tmem + kColS + wg * 64, ad, bd, kIdescQK, ks > 0 ? 1u : 0u);
-                }
+                });
                 tc_commit(bar(kBarSFull + wg));
-                flush_pv();   // P V of the previous slot, after S of this one: keeps the tensor pipe fed
+                mbar_arrive(bar(kBarEmpty + slot));   // this issuer's share of the slot's release (the P V commit is another)
+                flush_pv();   // P V of the previous own slot, after S of this one
                 pend_slot = slot;
-                pend_wg = wg;
                 pend_npg = npg;
                 pend_c = c;
-                cw[wg] = c + 1;
+                ++c;
             }
             flush_pv();
+            if (wg == 0) { TCPROF_FLUSH(0); }
         }
         __syncwarp();
     } else {
@@ -391,20 +424,24 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const float scale_log2 = a.scale_log2;
         const int G = a.G;
         float2* s_ml = reinterpret_cast<float2*>(smem + kMlOff);
-        const uint32_t p_row = sbase + kPOff + wg * kPBytes + row * 128;
 
         int cwg = 0;        // slots this warpgroup has processed (all items)
         int citem = 0;      // ... in the current item
         int item_k = -1;
         WorkItem it{};
         int rows = 0;
-        bool valid = false;
+        bool valid = false, warp_has_rows = false;
         int64_t mb = 0;
         float m = -INFINITY, l = 0.f;
+        TCPROF_DECL;
+#ifdef RKSC_WAIT_PROFILE
+        unsigned long long tcq[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        long long tcq_t = 0;
+#endif
 
         for (int seq = 0;; ++seq) {
             const int slot = seq % kNS;
-            wait_or_abort(bar(kBarFull + slot), (uint32_t)(seq / kNS) & 1u);
+            TCPROF_WAIT(1, wait_or_abort(bar(kBarFull + slot), (uint32_t)(seq / kNS) & 1u));
             if (*s_abort) break;
             const int4 hdr = *reinterpret_cast<const int4*>(&s_hdr[slot]);   // item, group, pages, last
             if (hdr.x < 0) break;
@@ -422,6 +459,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 ++item_k;
                 rows = it.num_sharers * G;
                 valid = row < rows;
+                warp_has_rows = quad * 32 < rows;
                 m = -INFINITY;
                 l = 0.f;
                 citem = 0;
@@ -450,9 +488,12 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 
             if ((g & 1) == wg) {
                 // ---- this warpgroup's slot: S row -> softmax -> P row ----
-                wait_or_abort(bar(kBarSFull + wg), (uint32_t)cwg & 1u);
+                TCPROF_WAIT(2, wait_or_abort(bar(kBarSFull + wg), (uint32_t)cwg & 1u));
                 if (*s_abort) break;
                 tc_fence_after();
+#ifdef RKSC_WAIT_PROFILE
+                tcq_t = clock64();
+#endif
                 uint32_t sr[2][32];
                 tmem_ld32(lane_addr + kColS + wg * 64, sr[0]);
                 tmem_ld32(lane_addr + kColS + wg * 64 + 32, sr[1]);
@@ -460,22 +501,41 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarSFree + wg));
+                TCPROF_MARK(0);
 
                 const int nvalid = it.num_tokens - g * kSlotTokens;   // tokens of this slot that exist
                 float mx = -INFINITY;
+#ifdef RKSC_TC_SKIP_SOFTMAX
+                mx = __uint_as_float(sr[0][0]) * 0.f;
+#else
+                if (warp_has_rows) {
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
+                    if (nvalid >= kSlotTokens) {
 #pragma unroll
-                for (int j = 0; j < 64; ++j) {
-                    float v = __uint_as_float(sr[j >> 5][j & 31]) * scale_log2;
-                    v = (j < nvalid) ? v : -INFINITY;
-                    sr[j >> 5][j & 31] = __float_as_uint(v);
-                    mx = fmaxf(mx, v);
+                        for (int j = 0; j < 64; ++j) {
+                            const float v = __uint_as_float(sr[j >> 5][j & 31]) * scale_log2;
+                            sr[j >> 5][j & 31] = __float_as_uint(v);
+                            mx4[j & 3] = fmaxf(mx4[j & 3], v);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 64; ++j) {
+                            float v = __uint_as_float(sr[j >> 5][j & 31]) * scale_log2;
+                            v = (j < nvalid) ? v : -INFINITY;
+                            sr[j >> 5][j & 31] = __float_as_uint(v);
+                            mx4[j & 3] = fmaxf(mx4[j & 3], v);
+                        }
+                    }
+                    mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 }
+#endif
                 const float m_new = valid ? fmaxf(m, mx) : m;
                 const bool grew = valid && (m_new > m);
+                TCPROF_MARK(1);
 
                 // the previous P V of this warpgroup must be complete before P is overwritten or O touched
                 if (citem > 0) {
-                    wait_or_abort(bar(kBarODone + wg), (uint32_t)(cwg - 1) & 1u);
+                    TCPROF_WAIT(3, wait_or_abort(bar(kBarODone + wg), (uint32_t)(cwg - 1) & 1u));
                     if (*s_abort) break;
                     tc_fence_after();
                     if (__any_sync(0xffffffffu, grew)) {
@@ -494,39 +554,46 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     }
                 }
                 m = m_new;
+                TCPROF_MARK(2);
 
                 float ps[4] = {0.f, 0.f, 0.f, 0.f};
+#ifndef RKSC_TC_SKIP_SOFTMAX
+                if (warp_has_rows) {
+                    const float mm = valid ? m : 0.f;   // rows past the item's end hold zeros: harmless, never read
 #pragma unroll
-                for (int j = 0; j < 64; ++j) {
-                    const float p = valid ? fast_exp2(__uint_as_float(sr[j >> 5][j & 31]) - m) : 0.f;
-                    sr[j >> 5][j & 31] = __float_as_uint(p);
-                    ps[j >> 4] += p;
+                    for (int j = 0; j < 64; ++j) {
+                        const float p = fast_exp2(__uint_as_float(sr[j >> 5][j & 31]) - mm);
+                        sr[j >> 5][j & 31] = __float_as_uint(p);
+                        ps[j >> 4] += p;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) sr[j >> 5][j & 31] = 0u;
                 }
+#endif
                 l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
                 if (valid && a.block_mass != nullptr) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
                         if (j < npg) a.block_mass[mb + g * 4 + j] = m + fast_log2(ps[j]);
                 }
-                // P row as bf16, 8 chunks of 8 tokens, 128-byte swizzled
+                TCPROF_MARK(3);
+                // P row as bf16 pairs into this warpgroup's P columns of tensor memory (A operand of P V)
+                {
+                    uint32_t pk[32];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    uint32_t w[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int j = c * 8 + 2 * e;
-                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(sr[j >> 5][j & 31]),
-                                                                        __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]));
-                        w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+                    for (int j = 0; j < 32; ++j) {
+                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(sr[(2 * j) >> 5][(2 * j) & 31]),
+                                                                        __uint_as_float(sr[(2 * j + 1) >> 5][(2 * j + 1) & 31]));
+                        pk[j] = *reinterpret_cast<const uint32_t*>(&b2);
                     }
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_row + ((c ^ (row & 7)) << 4)), "r"(w[0]),
-                                 "r"(w[1]), "r"(w[2]), "r"(w[3])
-                                 : "memory");
+                    tmem_st32(lane_addr + kColP + wg * 32, pk);
+                    tmem_wait_st();
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarPFull + wg));
+                TCPROF_MARK(4);
                 ++cwg;
                 ++citem;
             }
@@ -542,7 +609,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             s_ml[wg * 128 + row] = make_float2(m, l);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarEpiA));
-            wait_or_abort(bar(kBarEpiA), (uint32_t)item_k & 1u);
+            TCPROF_WAIT(4, wait_or_abort(bar(kBarEpiA), (uint32_t)item_k & 1u));
             if (*s_abort) break;
             tc_fence_after();
             {
@@ -587,9 +654,15 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarEpiB));
-            wait_or_abort(bar(kBarEpiB), (uint32_t)item_k & 1u);
+            TCPROF_WAIT(5, wait_or_abort(bar(kBarEpiB), (uint32_t)item_k & 1u));
             if (*s_abort) break;
         }
+#ifdef RKSC_WAIT_PROFILE
+        if (warp == 0 && lane == 0) {
+            tcp[6] = (unsigned long long)cwg; tcp[7] = (unsigned long long)(item_k + 1); TCPROF_FLUSH(8);
+            for (int _i = 0; _i < 8; ++_i) g_tc_prof[blockIdx.x + 128][_i] = tcq[_i];
+        }
+#endif
     }
 
     // ---- common exit: free the tensor memory once nobody uses it ----
@@ -602,6 +675,12 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 }
 
 }  // namespace
+
+#ifdef RKSC_WAIT_PROFILE
+extern "C" __attribute__((visibility("default"))) int rksc_debug_tc_profile(unsigned long long* host_out) {
+    return cudaMemcpyFromSymbol(host_out, g_tc_prof, sizeof(g_tc_prof)) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 size_t tc_kernel_smem_bytes() { return kSmemTotal + 1024; }
 
