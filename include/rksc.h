@@ -192,6 +192,38 @@ RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan* plan, cons
                                      void* workspace, size_t workspace_bytes,
                                      int32_t* device_status, void* stream, int32_t phases);
 
+/* ------------------------------------------------------------------------------------------
+ * rksc_branch_decode_attention_static: the same attention for callers that cannot allocate.
+ * (No counterpart in the paper: this is a packaging variant of the call above.)
+ *
+ * Some callers have no way to supply the workspace: a serving process that handed all device
+ * memory to its own pool at start-up and must not grow, a plug-in that is forbidden to call
+ * the allocating CUDA entry points, or a latency path that cannot afford the device-wide
+ * synchronisation an allocation may imply.  For them this entry point takes no workspace: the
+ * partial results go to a scratch array that is compiled into the library
+ * (RKSC_STATIC_WORKSPACE_BYTES of device memory on every GPU that loads the library, held
+ * until the process exits).  The call itself allocates and frees nothing, on the host side too
+ * it only launches kernels.  Inputs, outputs and device_status are passed as above; the plan
+ * was created beforehand with rksc_plan_create (that call does allocate).
+ *
+ *   - A plan that needs more than RKSC_STATIC_WORKSPACE_BYTES (see rksc_plan_query) is
+ *     refused with RKSC_ERR_WORKSPACE before anything is launched: use the call above.
+ *   - The first call on a device looks up the scratch array's device address (once per
+ *     device, with that device current) and keeps it.  Make that first call during set-up,
+ *     before any stream capture is begun on the device.
+ *   - Every call on a device uses the same scratch array.  Nothing in it has to start at
+ *     zero (each launch writes every partial row it later reads), so nothing is cleared and
+ *     the previous call's partials simply stay there until overwritten.  Two calls that may
+ *     overlap on the GPU (different streams, or different plans in flight together) race on
+ *     it: keep calls of this entry point ordered on one stream per device.
+ * Errors: as rksc_branch_decode_attention, plus RKSC_ERR_WORKSPACE as described.
+ * ------------------------------------------------------------------------------------------ */
+#define RKSC_STATIC_WORKSPACE_BYTES (16u << 20)
+RKSC_API int32_t rksc_branch_decode_attention_static(const rksc_plan* plan, const void* q,
+                                     const void* k_pool, const void* v_pool,
+                                     float* out, float* block_mass,
+                                     int32_t* device_status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -18,6 +18,8 @@ from .binding import (  # noqa: F401
     rksc_tables_from_gate,
     rksc_plan_create,
     rksc_branch_decode_attention,
+    rksc_branch_decode_attention_static,
+    STATIC_WORKSPACE_BYTES,
     split_block_mass,
     EXPORTED_SYMBOLS,
 )

@@ -28,7 +28,9 @@ EXPORTED_SYMBOLS = (
     "rksc_plan_destroy",
     "rksc_branch_decode_attention",
     "rksc_branch_decode_attention_phases",
+    "rksc_branch_decode_attention_static",
 )
+STATIC_WORKSPACE_BYTES = 16 << 20
 
 
 class RkscError(RuntimeError):
@@ -97,6 +99,8 @@ def lib() -> C.CDLL:
     L.rksc_branch_decode_attention.argtypes = [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p, C.c_void_p]
     L.rksc_branch_decode_attention_phases.restype = C.c_int32
     L.rksc_branch_decode_attention_phases.argtypes = [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p, C.c_void_p, C.c_int32]
+    L.rksc_branch_decode_attention_static.restype = C.c_int32
+    L.rksc_branch_decode_attention_static.argtypes = [C.c_void_p] * 8
     _lib = L
     return L
 
@@ -301,3 +305,18 @@ def split_block_mass(plan: Plan, block_mass) -> list:
         lo, hi = int(plan.mass_off[b]) * Hq, int(plan.mass_off[b + 1]) * Hq
         res.append(flat[lo:hi].reshape(Hq, -1) if hi > lo else np.zeros((Hq, 0), np.float32))
     return res
+
+
+def rksc_branch_decode_attention_static(plan: Plan, q, k_pool, v_pool, out, block_mass, device_status, stream=None):
+    """The attention for callers that may not allocate: no workspace argument, nothing is allocated here.
+
+    Every buffer is the caller's (``out`` fp32 [B][Hq][d], ``block_mass`` fp32 flat or None,
+    ``device_status`` int32 [1]); the partial results go to the scratch array compiled into the
+    library.  Plans needing more than STATIC_WORKSPACE_BYTES raise RkscError (status -4).  Calls
+    share that scratch, so keep them ordered on one stream per device."""
+    st = lib().rksc_branch_decode_attention_static(
+        plan._h, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), out.data_ptr(),
+        block_mass.data_ptr() if block_mass is not None else None,
+        device_status.data_ptr() if device_status is not None else None, _stream_ptr(stream))
+    _check(st, "rksc_branch_decode_attention_static")
+    return out, block_mass, device_status

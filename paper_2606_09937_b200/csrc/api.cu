@@ -322,3 +322,53 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
     }
     return RKSC_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Attention without any allocation by the caller: the partial-result scratch lives in the library
+// ---------------------------------------------------------------------------------------------
+
+namespace {
+
+// The scratch the segment kernels write their partial results to and the merge kernel reads them
+// from.  It is part of the loaded module: every GPU that loads this library keeps these bytes
+// until the process exits.
+static __device__ __align__(256) unsigned char g_static_workspace[RKSC_STATIC_WORKSPACE_BYTES];
+
+// In host code the array's name is only a handle for the runtime, not a device address; the address
+// the kernels need is asked for once per device and kept here.
+void* g_static_workspace_ptr[kMaxDevices];
+
+int32_t static_workspace(int dev, void** out) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_static_workspace_ptr[dev]) {
+        void* p = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&p, g_static_workspace);   // for the current device
+        if (e != cudaSuccess || !p) {
+            g_last_cuda = e;
+            cudaGetLastError();
+            return RKSC_ERR_CUDA;
+        }
+        g_static_workspace_ptr[dev] = p;
+    }
+    *out = g_static_workspace_ptr[dev];
+    return RKSC_OK;
+}
+
+}  // namespace
+
+extern "C" RKSC_API int32_t rksc_branch_decode_attention_static(const rksc_plan* plan, const void* q,
+                                                               const void* k_pool, const void* v_pool, float* out,
+                                                               float* block_mass, int32_t* device_status,
+                                                               void* stream) {
+    if (!plan) return RKSC_ERR_INVALID_ARG;
+    if (plan->host.workspace_bytes > (size_t)RKSC_STATIC_WORKSPACE_BYTES) return RKSC_ERR_WORKSPACE;
+    if (plan->host.B == 0) return RKSC_OK;
+    int dev = -1;
+    int32_t st = ensure_device(&dev);
+    if (st != RKSC_OK) return st;
+    void* ws = nullptr;
+    st = static_workspace(dev, &ws);
+    if (st != RKSC_OK) return st;
+    return rksc_branch_decode_attention(plan, q, k_pool, v_pool, out, block_mass, ws,
+                                        (size_t)RKSC_STATIC_WORKSPACE_BYTES, device_status, stream);
+}
