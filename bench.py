@@ -18,7 +18,6 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
 import threading
 import time
@@ -52,11 +51,12 @@ WORKLOAD_LABEL = {
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="batched_serving", choices=list(WORKLOAD_LABEL))
-    ap.add_argument("--cpu-sample-branches", type=int, default=96)
+    ap.add_argument("--cpu-sample-branches", type=int, default=0, help="branches the oracle runs (0 = the whole batch)")
+    ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-config attention-only table")
     ap.add_argument("--no-e2e", action="store_true")
@@ -77,55 +77,57 @@ def measured_peak_gbs():
 # ----------------------------------------------------------------------------------------------
 
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons through NVML from a thread while the timed region runs."""
 
-    def __init__(self, index: int):
-        self.index = index
-        self.proc = None
-        self.lines = []
-        self.thread = None
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
+               "hw_thermal_slowdown": 0x40, "hw_power_brake_slowdown": 0x80}
+
+    def __init__(self, torch_device):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            uuid = getattr(torch.cuda.get_device_properties(torch_device), "uuid", None)
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(torch_device.index or 0)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for name, bit in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except Exception:
-            self.proc = None
-            return
-        self.thread = threading.Thread(target=self._read, daemon=True)
-        self.thread.start()
-
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            parts = [p.strip() for p in ln.split(",")]
-            if len(parts) < 6:
-                continue
-            try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, parts[2:6]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -253,7 +255,7 @@ def oracle_pass(w, sample_branches: int):
         tt = w.tables
         t = {k: getattr(tt, k) for k in ("seg_block_off", "seg_blocks", "seg_num_tokens", "br_seg_off", "br_segs")}
     B = len(t["br_seg_off"]) - 1
-    nb = min(B, max(1, sample_branches))
+    nb = B if sample_branches <= 0 else min(B, sample_branches)
     oracle.branch_decode_attention(L.num_q_heads, L.num_kv_heads, L.head_dim, L.sm_scale,
                                    t["seg_block_off"], t["seg_blocks"], t["seg_num_tokens"],
                                    t["br_seg_off"], t["br_segs"], q, kp, vp, branches=range(nb))
@@ -277,7 +279,7 @@ def run_reference(args):
             times.append(dt)
     t = sum(times) / len(times)
     val = ub / t / 1e12
-    sample = f"first {nb} of {B} branches of the batch (gate over all branches, attention over the sample)"
+    sample = f"{nb} of {B} branches of the batch per step (gate over all branches, attention over these)"
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
@@ -334,7 +336,7 @@ def run_ours(args):
     kv_bytes, alg_bytes = algorithmic_bytes(plan, w.layout)
     small = kv_bytes < 2 * l2_bytes   # then L2 must be flushed between timed iterations
 
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(dev)
     if rank == 0:
         sampler.start()
     seg_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
@@ -355,13 +357,8 @@ def run_ours(args):
     step_ms = [a.elapsed_time(b) for a, b in step_ev]
     seg_ms = [a.elapsed_time(b) for a, b in seg_ev]
     total_ms = sum(step_ms)           # device time of exactly K steps (flushes excluded)
-    tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-    total_ms_max = float(tt.item())
     assert int(batch.status.item()) == 0, "a kernel reported a device-side timeout"
-
-    value = world * kv_bytes * args.steps / (total_ms_max * 1e-3) / 1e12
+    value, total_ms_max = aggregate_over_ranks(dist, dev, kv_bytes, args.steps, total_ms)
     peak_gbs, peak_kind = measured_peak_gbs()
     seg_avg_ms = sum(seg_ms) / len(seg_ms)
     achieved = alg_bytes / (seg_avg_ms * 1e-3) / 1e9
@@ -385,7 +382,7 @@ def run_ours(args):
         "wall_ms_per_step": t_wall * 1e3 / args.steps,
         "gpu_launches": launches,
         "roofline": {
-            "kernel": "seg_attn_warp_kernel", "bound": "hbm", "achieved": achieved, "peak": peak_gbs,
+            "kernel": "segment attention: seg_attn_tc_kernel + seg_attn_warp_kernel (chained launches)", "bound": "hbm", "achieved": achieved, "peak": peak_gbs,
             "unit": "GB/s", "frac": achieved / peak_gbs, "peak_source": peak_kind,
             "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": seg_avg_ms,
             "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
@@ -403,18 +400,74 @@ def run_ours(args):
             "pct_of_measured_copy_peak": 100.0 * kv_bytes / (med * 1e-3) / 1e9 / peak_gbs,
             "branch_steps_per_s": B / (med * 1e-3),
         }
+        if not args.no_e2e and batch.has_gate:
+            line["e2e"] = run_e2e(rk, batch, kv_bytes, args.e2e_steps)
         if not args.no_sweep:
             line["configs"] = sweep_configs(rk, dev, flush, peak_gbs, skip=args.workload, cached=(args.workload, line))
         if not args.no_cpu_baseline:
             dt, ub, cores, nb, Bt = oracle_pass(w, args.cpu_sample_branches)
             line["cpu_baseline"] = {
                 "value": ub / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
-                "sample": f"first {nb} of {Bt} branches of the batch (gate over all, attention over the sample), "
-                          f"{dt:.1f} s", "seconds": dt}
+                "sample": f"{nb} of {Bt} branches of the batch (gate over all branches, attention over these), "
+                          f"one pass, {dt:.1f} s", "seconds": dt}
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_e2e(rk, batch: DeviceBatch, kv_bytes: int, steps: int):
+    """The metric through rksc_decode_step_host: per-step inputs in pinned host memory, results read back.
+
+    The KV pool stays resident (it is device state written by earlier decode steps); hidden states,
+    candidate ids, page lists and queries go host -> device and map, sigma, out and block masses come
+    back inside every timed step."""
+    import torch
+    w = batch.w
+    g, L = w.gate, w.layout
+    B = w.num_branches
+    hb = g.h_branch.pin_memory()
+    hr = g.h_root.pin_memory()
+    q = w.q.pin_memory()
+    m_host = torch.empty(B, dtype=torch.int32).pin_memory()
+    s_host = torch.empty(B, dtype=torch.float32).pin_memory()
+    out_host = torch.empty((B, L.num_q_heads, L.head_dim), dtype=torch.float32).pin_memory()
+    mass_host = torch.empty(max(batch.mass.numel(), 1), dtype=torch.float32).pin_memory()
+    mass_off = np.zeros(B + 1, dtype=np.int64)
+
+    def one():
+        rk.rksc_decode_step_host(L, hb, hr, g.cand_prefix, g.alpha, g.tau, w.flat, q, batch.k_pool, batch.v_pool,
+                                 m_host, s_host, out_host, mass_host, mass_off)
+    for _ in range(3):
+        one()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    e1.synchronize()
+    wall = time.perf_counter() - t0
+    ms = e0.elapsed_time(e1) / steps
+    mass_elems = int(mass_off[-1]) * L.num_q_heads
+    h2d = hb.numel() * 4 + hr.numel() * 4 + B * 4 + q.numel() * 2
+    d2h = B * 4 * 2 + out_host.numel() * 4 + mass_elems * 4 + 4
+    return {"value": kv_bytes / (ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "ms_per_step": ms, "wall_ms_per_step": wall * 1e3 / steps,
+            "call": "rksc_decode_step_host (pinned host buffers; KV pool resident in HBM)", "steps": steps}
+
+
+def aggregate_over_ranks(dist, dev, kv_bytes: int, steps: int, total_ms: float):
+    """Whole-job throughput: bytes summed over ranks (each rank has its own batch), time = max over ranks."""
+    import torch
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    b = torch.tensor([float(kv_bytes)], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    total_ms_max = float(t.item())
+    return float(b.item()) * steps / (total_ms_max * 1e-3) / 1e12, total_ms_max
 
 
 def punch_long_context(rk, batch: DeviceBatch):

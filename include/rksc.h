@@ -193,6 +193,33 @@ RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan* plan, cons
                                      int32_t* device_status, void* stream, int32_t phases);
 
 /* ------------------------------------------------------------------------------------------
+ * rksc_decode_step_host: the whole path (gate -> tables -> plan -> attention) in one call for a
+ * caller whose per-step data lives in host memory (paper Algorithm 1 lines 2-4 restricted to the
+ * ASKS gate and the attention of one decode step of one layer).
+ *
+ * Host inputs (pinned memory makes the copies asynchronous): h_branch [B][L][D], h_root [P][L][D]
+ * fp32, cand_prefix [B], the three page-list CSRs of rksc_tables_from_gate, q [B][Hq][d] bf16.
+ * Device inputs: the resident KV pool (k_pool, v_pool) - a KV cache is device state written by
+ * earlier steps, not a per-step input.
+ * Host outputs: branch_to_prefix [B], sigma [B] (may be NULL), out [B][Hq][d] fp32, block_mass
+ * (may be NULL; capacity in floats, RKSC_ERR_INVALID_ARG if smaller than the plan's mass_elems),
+ * mass_off [B+1] (may be NULL).
+ * The call allocates its device scratch stream-ordered (cudaMallocAsync / cudaFreeAsync on
+ * `stream`), synchronises the stream twice (after the gate, and at the end), and returns the
+ * status of the first failing stage or the device_status word of the attention.
+ * ------------------------------------------------------------------------------------------ */
+RKSC_API int32_t rksc_decode_step_host(
+    const rksc_layout* layout,
+    const float* h_branch, const float* h_root, const int32_t* cand_prefix,
+    int32_t B, int32_t P, int32_t L, int32_t D, float alpha, float tau,
+    const int32_t* shared_off, const int32_t* shared_pages, const int32_t* shared_ntok,
+    const int32_t* priv_off,   const int32_t* priv_pages,   const int32_t* priv_ntok,
+    const int32_t* sfx_off,    const int32_t* sfx_pages,    const int32_t* sfx_ntok,
+    const void* q, const void* k_pool, const void* v_pool,
+    int32_t* branch_to_prefix, float* sigma, float* out, float* block_mass,
+    int64_t block_mass_capacity, int64_t* mass_off, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * rksc_branch_decode_attention_static: the same attention for callers that cannot allocate.
  * (No counterpart in the paper: this is a packaging variant of the call above.)
  *

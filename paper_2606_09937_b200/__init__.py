@@ -19,6 +19,7 @@ from .binding import (  # noqa: F401
     rksc_plan_create,
     rksc_branch_decode_attention,
     rksc_branch_decode_attention_static,
+    rksc_decode_step_host,
     STATIC_WORKSPACE_BYTES,
     split_block_mass,
     EXPORTED_SYMBOLS,

@@ -29,6 +29,7 @@ EXPORTED_SYMBOLS = (
     "rksc_branch_decode_attention",
     "rksc_branch_decode_attention_phases",
     "rksc_branch_decode_attention_static",
+    "rksc_decode_step_host",
 )
 STATIC_WORKSPACE_BYTES = 16 << 20
 
@@ -99,6 +100,10 @@ def lib() -> C.CDLL:
     L.rksc_branch_decode_attention.argtypes = [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p, C.c_void_p]
     L.rksc_branch_decode_attention_phases.restype = C.c_int32
     L.rksc_branch_decode_attention_phases.argtypes = [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p, C.c_void_p, C.c_int32]
+    L.rksc_decode_step_host.restype = C.c_int32
+    L.rksc_decode_step_host.argtypes = ([C.POINTER(_CLayout), C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 4 +
+                                        [C.c_float, C.c_float] + [i32p] * 9 + [C.c_void_p] * 7 +
+                                        [C.c_int64, C.c_void_p, C.c_void_p])
     L.rksc_branch_decode_attention_static.restype = C.c_int32
     L.rksc_branch_decode_attention_static.argtypes = [C.c_void_p] * 8
     _lib = L
@@ -320,3 +325,31 @@ def rksc_branch_decode_attention_static(plan: Plan, q, k_pool, v_pool, out, bloc
         device_status.data_ptr() if device_status is not None else None, _stream_ptr(stream))
     _check(st, "rksc_branch_decode_attention_static")
     return out, block_mass, device_status
+
+
+def rksc_decode_step_host(layout, h_branch, h_root, cand_prefix, alpha, tau, flat, q, k_pool, v_pool,
+                          branch_to_prefix, sigma, out, block_mass, mass_off=None, stream=None):
+    """The whole path for host-resident per-step data (see rksc_decode_step_host in rksc.h).
+
+    h_branch, h_root, q, branch_to_prefix, sigma, out, block_mass are HOST torch tensors (pinned for
+    asynchronous copies); cand_prefix and the page lists (``flat``: an object with the nine CSR arrays
+    and num_prefixes) are host int32 arrays; k_pool / v_pool are the device-resident pool.
+    Returns the status word (0 = ok)."""
+    lay = layout if isinstance(layout, Layout) else Layout.of(layout)
+    B, L, D = h_branch.shape
+    P = h_root.shape[0]
+    cand = _i32(cand_prefix)
+    lists = [_i32(getattr(flat, n)) for n in ("shared_off", "shared_pages", "shared_ntok", "priv_off", "priv_pages",
+                                              "priv_ntok", "sfx_off", "sfx_pages", "sfx_ntok")]
+    mo = None
+    if mass_off is not None:
+        assert mass_off.dtype == np.int64 and mass_off.shape[0] == B + 1
+        mo = mass_off.ctypes.data
+    st = lib().rksc_decode_step_host(
+        C.byref(lay.c), h_branch.data_ptr(), h_root.data_ptr(), cand.ctypes.data, B, P, L, D, float(alpha), float(tau),
+        *[_p(a) for a in lists], q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(),
+        branch_to_prefix.data_ptr(), sigma.data_ptr() if sigma is not None else None, out.data_ptr(),
+        block_mass.data_ptr() if block_mass is not None else None,
+        block_mass.numel() if block_mass is not None else 0, mo, _stream_ptr(stream))
+    _check(st, "rksc_decode_step_host")
+    return st

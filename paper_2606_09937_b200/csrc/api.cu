@@ -324,6 +324,105 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
 }
 
 // ---------------------------------------------------------------------------------------------
+// The whole path for host-resident inputs (KV pool resident on the device)
+// ---------------------------------------------------------------------------------------------
+
+namespace {
+
+struct AsyncBuf {   // stream-ordered device buffer, released on scope exit
+    void* p = nullptr;
+    cudaStream_t s = nullptr;
+    cudaError_t alloc(size_t bytes, cudaStream_t stream) {
+        s = stream;
+        return cudaMallocAsync(&p, bytes ? bytes : 16, stream);
+    }
+    ~AsyncBuf() {
+        if (p) cudaFreeAsync(p, s);
+    }
+};
+
+}  // namespace
+
+extern "C" RKSC_API int32_t rksc_decode_step_host(
+    const rksc_layout* layout, const float* h_branch, const float* h_root, const int32_t* cand_prefix, int32_t B,
+    int32_t P, int32_t L, int32_t D, float alpha, float tau, const int32_t* shared_off, const int32_t* shared_pages,
+    const int32_t* shared_ntok, const int32_t* priv_off, const int32_t* priv_pages, const int32_t* priv_ntok,
+    const int32_t* sfx_off, const int32_t* sfx_pages, const int32_t* sfx_ntok, const void* q, const void* k_pool,
+    const void* v_pool, int32_t* branch_to_prefix, float* sigma, float* out, float* block_mass,
+    int64_t block_mass_capacity, int64_t* mass_off, void* stream) {
+    if (!layout || !h_branch || !h_root || !cand_prefix || !q || !k_pool || !v_pool || !branch_to_prefix || !out)
+        return RKSC_ERR_INVALID_ARG;
+    if (B <= 0 || P <= 0 || L <= 0 || D <= 0) return RKSC_ERR_INVALID_ARG;
+    int32_t st = ensure_device(nullptr);
+    if (st != RKSC_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t nb = (size_t)B * L * D * sizeof(float), nr = (size_t)P * L * D * sizeof(float);
+    const size_t nq = (size_t)B * layout->num_q_heads * layout->head_dim * 2;
+    const size_t nout = (size_t)B * layout->num_q_heads * layout->head_dim * sizeof(float);
+    AsyncBuf d_hb, d_hr, d_cand, d_map, d_sigma, d_q, d_out, d_mass, d_ws, d_status;
+    cudaError_t e = cudaSuccess;
+    auto ok = [&](cudaError_t r) {
+        if (e == cudaSuccess && r != cudaSuccess) e = r;
+        return e == cudaSuccess;
+    };
+    auto fail = [&]() {
+        g_last_cuda = e;
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    };
+    // gate: inputs to the device, kernel, map (and sigma) back
+    if (!ok(d_hb.alloc(nb, s)) || !ok(d_hr.alloc(nr, s)) || !ok(d_cand.alloc((size_t)B * 4, s)) ||
+        !ok(d_map.alloc((size_t)B * 4, s)) || !ok(d_sigma.alloc((size_t)B * 4, s)) || !ok(d_q.alloc(nq, s)) ||
+        !ok(d_out.alloc(nout, s)) || !ok(d_status.alloc(16, s)))
+        return fail();
+    ok(cudaMemcpyAsync(d_hb.p, h_branch, nb, cudaMemcpyHostToDevice, s));
+    ok(cudaMemcpyAsync(d_hr.p, h_root, nr, cudaMemcpyHostToDevice, s));
+    ok(cudaMemcpyAsync(d_cand.p, cand_prefix, (size_t)B * 4, cudaMemcpyHostToDevice, s));
+    ok(cudaMemcpyAsync(d_q.p, q, nq, cudaMemcpyHostToDevice, s));
+    ok(cudaMemsetAsync(d_status.p, 0, 16, s));
+    if (e != cudaSuccess) return fail();
+    st = rksc_asks_gate((const float*)d_hb.p, (const float*)d_hr.p, (const int32_t*)d_cand.p, B, P, L, D, alpha, tau,
+                        (int32_t*)d_map.p, (float*)d_sigma.p, stream);
+    if (st != RKSC_OK) return st;
+    ok(cudaMemcpyAsync(branch_to_prefix, d_map.p, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
+    if (sigma) ok(cudaMemcpyAsync(sigma, d_sigma.p, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
+    ok(cudaStreamSynchronize(s));   // the tables are built on the host from the map
+    if (e != cudaSuccess) return fail();
+
+    rksc_tables tables;
+    st = rksc_tables_from_gate(B, P, branch_to_prefix, shared_off, shared_pages, shared_ntok, priv_off, priv_pages,
+                               priv_ntok, sfx_off, sfx_pages, sfx_ntok, &tables);
+    if (st != RKSC_OK) return st;
+    rksc_plan* plan = nullptr;
+    st = rksc_plan_create(layout, &tables, &plan);
+    rksc_tables_free(&tables);
+    if (st != RKSC_OK) return st;
+    const HostPlan& H = plan->host;
+    if (mass_off) std::memcpy(mass_off, H.mass_off.data(), (size_t)(B + 1) * sizeof(int64_t));
+    if (block_mass && block_mass_capacity < H.mass_elems) {
+        rksc_plan_destroy(plan);
+        return RKSC_ERR_INVALID_ARG;
+    }
+    if (!ok(d_ws.alloc(H.workspace_bytes, s)) || (block_mass && !ok(d_mass.alloc((size_t)H.mass_elems * 4, s)))) {
+        rksc_plan_destroy(plan);
+        return fail();
+    }
+    st = rksc_branch_decode_attention(plan, d_q.p, k_pool, v_pool, (float*)d_out.p, block_mass ? (float*)d_mass.p : nullptr,
+                                      d_ws.p, H.workspace_bytes, (int32_t*)d_status.p, stream);
+    int32_t dev_status = 0;
+    if (st == RKSC_OK) {
+        ok(cudaMemcpyAsync(out, d_out.p, nout, cudaMemcpyDeviceToHost, s));
+        if (block_mass) ok(cudaMemcpyAsync(block_mass, d_mass.p, (size_t)H.mass_elems * 4, cudaMemcpyDeviceToHost, s));
+        ok(cudaMemcpyAsync(&dev_status, d_status.p, 4, cudaMemcpyDeviceToHost, s));
+    }
+    ok(cudaStreamSynchronize(s));   // also ends the plan's use before it is destroyed
+    rksc_plan_destroy(plan);
+    if (st != RKSC_OK) return st;
+    if (e != cudaSuccess) return fail();
+    return dev_status;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Attention without any allocation by the caller: the partial-result scratch lives in the library
 // ---------------------------------------------------------------------------------------------
 

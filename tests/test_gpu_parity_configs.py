@@ -1,0 +1,101 @@
+"""CUDA path vs the oracle on the five configurations at full size, in the launch setup bench.py times.
+
+Small configs are compared element by element; on the large ones the oracle computes a sample of
+branches one by one (every sampled branch is compared in full), and properties that hold at any size
+(masses sum to 1, finite outputs) are checked for all branches.
+"""
+import numpy as np
+import pytest
+
+import workloads
+from helpers import (MASS_SUM_ATOL, check_attention, cuda_attention, cuda_gate, oracle_attention,
+                     oracle_gate, oracle_tables_from_map)
+
+pytestmark = pytest.mark.gpu
+
+
+def _all_branch_properties(out, masses):
+    assert np.isfinite(out).all()
+    for m in masses:
+        if m.size:
+            assert np.isfinite(m).all() and (m >= 0).all()
+            assert np.abs(m.astype(np.float64).sum(axis=1) - 1.0).max() <= MASS_SUM_ATOL
+
+
+def _gate_and_tables(w):
+    import paper_2606_09937_b200 as rk
+    m_ref, s_ref = oracle_gate(w.gate)
+    assert np.abs(s_ref - np.float32(w.gate.tau)).min() >= 1e-3       # inputs keep clear of tau
+    m, s = cuda_gate(w.gate)
+    assert np.array_equal(m, m_ref)                                    # bit-exact map
+    assert np.abs(s - s_ref).max() < 1e-5
+    f = w.flat
+    t = rk.rksc_tables_from_gate(m, f.num_prefixes, f.shared_off, f.shared_pages, f.shared_ntok,
+                                 f.priv_off, f.priv_pages, f.priv_ntok, f.sfx_off, f.sfx_pages, f.sfx_ntok)
+    t_ref = oracle_tables_from_map(w, m_ref)
+    for k, v in t.as_dict().items():
+        assert np.array_equal(v, t_ref[k]), k                          # bit-exact tables
+    return t_ref
+
+
+def test_config1_tiny_full():
+    w = workloads.make_config("tiny")
+    t = _gate_and_tables(w)
+    for tables in (w.tables, t):          # as stated (4 sharers) and end to end (3 sharers + private copy)
+        ref_out, ref_m = oracle_attention(w, tables)
+        out, m, _ = cuda_attention(w, tables)
+        check_attention(out, m, ref_out, ref_m)
+
+
+def test_config2_qwen_layer_full():
+    w = workloads.make_config("qwen_layer")
+    t = _gate_and_tables(w)
+    ref_out, ref_m = oracle_attention(w, t)
+    out, m, plan = cuda_attention(w, t)
+    check_attention(out, m, ref_out, ref_m)
+    assert plan.unique_kv_tokens * w.layout.bytes_per_token == 8 << 20
+
+
+def test_config3_tot_full():
+    w = workloads.make_config("tot")
+    out, m, plan = cuda_attention(w)
+    _all_branch_properties(out, m)
+    assert plan.unique_kv_tokens == 22528 and plan.duplicated_kv_tokens == 114688
+    sample = [0, 1, 5, 17, 31, 42, 63]
+    ref_out, ref_m = oracle_attention(w, branches=sample)
+    check_attention(out, m, ref_out, ref_m, branches=sample)
+
+
+def test_config4_batched_serving_full():
+    w = workloads.make_config("batched_serving")
+    t = _gate_and_tables(w)
+    m_ref = np.where(w.gate.built_below_tau, -1, w.gate.cand_prefix)
+    assert int((m_ref < 0).sum()) == 77
+    out, m, plan = cuda_attention(w, t)
+    _all_branch_properties(out, m)
+    rng = np.random.default_rng(7)
+    priv = np.flatnonzero(w.gate.built_below_tau)
+    shared = np.flatnonzero(~w.gate.built_below_tau)
+    sample = sorted(set(rng.choice(priv, 6, replace=False).tolist() + rng.choice(shared, 10, replace=False).tolist()))
+    ref_out, ref_m = oracle_attention(w, t, branches=sample)
+    check_attention(out, m, ref_out, ref_m, branches=sample)
+
+
+def test_config5_long_context_with_holes_full():
+    w = workloads.make_config("long_context")
+    # eviction choice from the ORACLE's prior-step masses on three sampled branches x all heads,
+    # so that both sides get the same holed table and no oracle input comes from the GPU
+    prior = [0, 7, 15]
+    _, pm = oracle_attention(w, branches=prior)
+    npg = int(w.tables.seg_block_off[1])
+    scores = sum(pm[b][:, :npg].sum(axis=0) for b in prior)
+    ev = workloads.lowest_mass_pages(scores, 0.2)
+    assert len(ev) == 409
+    h = workloads.punch_holes(w, 0, ev)
+    assert int(h.tables.seg_block_off[1]) == 1639
+    out, m, plan = cuda_attention(h)
+    _all_branch_properties(out, m)
+    assert plan.unique_kv_tokens == 1639 * 16 + 16 * 2048
+    sample = [0, 9, 15]
+    ref_out, ref_m = oracle_attention(h, branches=sample)
+    check_attention(out, m, ref_out, ref_m, branches=sample)
