@@ -5,9 +5,10 @@
 // 128 rows of one MMA tile; a KV page staged in shared memory once then serves every sharing
 // branch (the shared-prefix read that replaces the paper's per-branch copies of the prefix cache,
 // Algorithm 1 line 3 / Section 2.2).  Here the product really is a dense contraction:
-//   S[128 x 64]  = Q[128 x d] K^T        (tcgen05.mma, A and B K-major in 128-byte-swizzled smem)
+//   S[128 x 64]  = Q[128 x d] K^T        (tcgen05.mma, A = Q read from tensor memory, B = K slot, K-major,
+//                                         in 128-byte-swizzled smem)
 //   O[128 x d]  += P[128 x 64] V         (A = P read from tensor memory, B = V MN-major in smem)
-// with S, P and O in tensor memory.  One persistent CTA per SM, eleven warps:
+// with Q, S, P and O in tensor memory.  One persistent CTA per SM, eleven warps:
 //   warps 0-3 / 4-7  two softmax warpgroups; thread = one stacked row (TMEM lane).  They take
 //                    alternate 64-token slots of an item, each with its own S and O accumulator and
 //                    its own running (max, sum), merged at the end of the item.  Per slot: tcgen05.ld
@@ -36,14 +37,12 @@ constexpr int kSmWarps = 8;                       // softmax warps (two warpgrou
 constexpr int kProducerWarp = kSmWarps;           // 8
 constexpr int kMmaWarp = kSmWarps + 1;            // 9 and 10: MMA issuers of warpgroup 0 and 1
 constexpr int kTcThreads = (kSmWarps + 3) * 32;   // 352
-constexpr int kNS = 5;                            // ring slots
+constexpr int kNS = 6;                            // ring slots
 constexpr int kSlotTokens = 64;                   // 4 pages
 constexpr int kKBytes = kSlotTokens * HD * 2;     // K (or V) of a slot: [half][64 tokens][128 B] = 16 KiB
 constexpr int kSlotBytes = 2 * kKBytes;
-constexpr int kRingBytes = kNS * kSlotBytes;      // 160 KiB
-constexpr int kQOff = kRingBytes;                 // Q tile [half][128 rows][128 B]
-constexpr int kQBytes = 128 * HD * 2;             // 32 KiB
-constexpr int kMlOff = kQOff + kQBytes;           // (m, l) exchange [2][128] float2
+constexpr int kRingBytes = kNS * kSlotBytes;      // 192 KiB
+constexpr int kMlOff = kRingBytes;                // (m, l) exchange [2][128] float2
 constexpr int kBarOff = kMlOff + 2 * 128 * 8;
 // mbarriers
 constexpr int kBarFull = 0;                       // [kNS]  producer -> everyone: slot landed (+ header)
@@ -52,7 +51,7 @@ constexpr int kBarSFull = kBarEmpty + kNS;        // [2]    S of the warpgroup's
 constexpr int kBarSFree = kBarSFull + 2;          // [2]    the warpgroup has copied S to registers
 constexpr int kBarPFull = kBarSFree + 2;          // [2]    P of the slot is in tensor memory
 constexpr int kBarODone = kBarPFull + 2;          // [2]    P V of the slot has completed
-constexpr int kBarQFull = kBarODone + 2;          // Q tile of the item is in shared memory
+constexpr int kBarQFull = kBarODone + 2;          // Q tile of the item is in tensor memory
 constexpr int kBarEpiA = kBarQFull + 1;           // item epilogue: (m, l) published
 constexpr int kBarEpiB = kBarEpiA + 1;            // item epilogue: accumulators read
 constexpr int kNumBars = kBarEpiB + 1;
@@ -64,6 +63,8 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0;                     // S[wg]: 64 fp32 columns at 64*wg
 constexpr uint32_t kColO = 128;                   // O[wg]: 128 fp32 columns at 128 + 128*wg
 constexpr uint32_t kColP = 384;                   // P[wg]: 64 bf16 = 32 columns at 384 + 32*wg
+constexpr uint32_t kColQ = 448;                   // Q: 128 bf16 per row = 64 columns (half wg written by warpgroup wg)
+constexpr float kRescaleStep = 8.f;               // O is rescaled only when a row's max moved by more than 2^8
 
 struct __align__(16) SlotHeader {
     int32_t item;        // index of the work item, -1: no more work
@@ -148,16 +149,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint
 __host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
            ((uint32_t)(128 >> 4) << 24);
-}
-__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-        "}\n"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
 }
 // A operand (128 x 16 bf16, two values per 32-bit column) read from tensor memory
 __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -279,15 +270,16 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         auto fetch_ids = [&](const WorkItem& w, int first) {
             return (first + lane < w.num_pages) ? __ldg(a.plan.seg_blocks + w.page_begin + first + lane) : 0;
         };
+        // One item is claimed ahead of the one being streamed (its descriptor and first page ids are
+        // fetched while this one streams); claiming further ahead would starve other CTAs, there
+        // being only a few of these long items per CTA.
         int seq = 0;
         int idx = claim();
         WorkItem it = fetch_item(idx);
         int ids = fetch_ids(it, 0);
-        int nidx = claim();
-        WorkItem nit = fetch_item(nidx);
-        int nids = fetch_ids(nit, 0);
         while (idx < a.num_tc_items && !*s_abort) {
-            const int nnidx = claim();
+            const int nidx = claim();
+            const WorkItem nit = fetch_item(nidx);
             const int ngroups = (it.num_pages + 3) / 4;
             int ids_ahead = 0;
             for (int g = 0; g < ngroups; ++g, ++seq) {
@@ -324,10 +316,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             }
             idx = nidx;
             it = nit;
-            ids = nids;
-            nidx = nnidx;
-            nit = fetch_item(nidx);
-            nids = fetch_ids(nit, 0);
+            ids = fetch_ids(it, 0);
         }
         {   // end marker
             const int slot = seq % kNS;
@@ -398,11 +387,10 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (c > 0) TCPROF_WAIT(2, wait_or_abort(bar(kBarSFree + wg), (uint32_t)(c - 1) & 1u));
                 if (*s_abort) break;
                 tc_fence_after();
-                const uint32_t qbase = sbase + kQOff, kbase = sbase + slot * kSlotBytes;
+                const uint32_t kbase = sbase + slot * kSlotBytes;
                 TCPROF_WAIT(5, for (int ks = 0; ks < HD / 16; ++ks) {
-                    const uint64_t ad = smem_desc(qbase + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
                     const uint64_t bd = smem_desc(kbase + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
-                    umma(tmem + kColS + wg * 64, ad, bd, kIdescQK, ks > 0 ? 1u : 0u);
+                    umma_ts(tmem + kColS + wg * 64, tmem + kColQ + ks * 8, bd, kIdescQK, ks > 0 ? 1u : 0u);
                 });
                 tc_commit(bar(kBarSFull + wg));
                 mbar_arrive(bar(kBarEmpty + slot));   // this issuer's share of the slot's release (the P V commit is another)
@@ -471,17 +459,23 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     qsrc = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) +
                                                           ((size_t)sh.branch * a.Hq + h) * HD + wg * 64);
                 }
-                // this warpgroup stages half `wg` (64 of the 128 dims) of every row, 128-byte swizzled
-                const uint32_t qdst = sbase + kQOff + wg * 16384 + row * 128;
+                // this warpgroup stages half `wg` (64 of the 128 dims) of every row into the Q columns of
+                // tensor memory: thread = row = TMEM lane, two bf16 per 32-bit column (A operand of Q K^T)
+                {
+                    uint32_t qr[32];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (valid) v = __ldg(qsrc + c);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(qdst + ((c ^ (row & 7)) << 4)), "r"(v.x),
-                                 "r"(v.y), "r"(v.z), "r"(v.w)
-                                 : "memory");
+                    for (int c = 0; c < 8; ++c) {
+                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                        if (valid) v = __ldg(qsrc + c);
+                        qr[4 * c] = v.x;
+                        qr[4 * c + 1] = v.y;
+                        qr[4 * c + 2] = v.z;
+                        qr[4 * c + 3] = v.w;
+                    }
+                    tmem_st32(lane_addr + kColQ + wg * 32, qr);
+                    tmem_wait_st();
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarQFull));
             }
@@ -529,17 +523,21 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 }
 #endif
-                const float m_new = valid ? fmaxf(m, mx) : m;
-                const bool grew = valid && (m_new > m);
                 TCPROF_MARK(1);
 
-                // the previous P V of this warpgroup must be complete before P is overwritten or O touched
-                if (citem > 0) {
+                // Running maximum with slack: m is raised (and O, l rescaled) only when a row's maximum
+                // moved up by more than kRescaleStep, so p = 2^(s - m) stays below 2^kRescaleStep and the
+                // TMEM round trip of O is rare.  The first slot of the item just adopts its maximum.
+                if (citem == 0) {
+                    if (valid) m = mx;
+                } else {
+                    // the previous P V of this warpgroup must be complete before P is overwritten or O touched
                     TCPROF_WAIT(3, wait_or_abort(bar(kBarODone + wg), (uint32_t)(cwg - 1) & 1u));
                     if (*s_abort) break;
                     tc_fence_after();
+                    const bool grew = valid && (mx > m + kRescaleStep);
                     if (__any_sync(0xffffffffu, grew)) {
-                        const float alpha = grew ? fast_exp2(m - m_new) : 1.f;
+                        const float alpha = grew ? fast_exp2(m - mx) : 1.f;
                         l *= alpha;
 #pragma unroll 1
                         for (int c = 0; c < HD / 32; ++c) {
@@ -551,9 +549,9 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                             tmem_st32(lane_addr + kColO + wg * 128 + c * 32, o);
                         }
                         tmem_wait_st();
+                        if (grew) m = mx;
                     }
                 }
-                m = m_new;
                 TCPROF_MARK(2);
 
                 float ps[4] = {0.f, 0.f, 0.f, 0.f};
