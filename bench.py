@@ -162,7 +162,12 @@ class DeviceBatch:
         self.out = torch.empty(tuple(self.q.shape), dtype=torch.float32, device=dev)
         self.mass = None
         self.workspace = None
-        self.tables = w.tables
+        self.tables = None
+        import paper_2606_09937_b200 as rk
+        self.layout = rk.Layout.of(w.layout)
+        self.lists = rk.GateLists(w.flat) if self.has_gate else None
+        if w.tables is not None:
+            self.tables = rk.Tables.of(w.tables)
 
     def ensure_buffers(self, plan):
         import torch
@@ -182,13 +187,9 @@ def run_step(rk, batch: DeviceBatch, seg_events=None):
                           branch_to_prefix=batch.map_dev, sigma=batch.sigma_dev)
         launches += 1
         batch.map_host.copy_(batch.map_dev, non_blocking=False)   # the host needs the map to build tables
-        tables = rk.rksc_tables_from_gate(batch.map_host.numpy(), f.num_prefixes,
-                                          f.shared_off, f.shared_pages, f.shared_ntok,
-                                          f.priv_off, f.priv_pages, f.priv_ntok,
-                                          f.sfx_off, f.sfx_pages, f.sfx_ntok)
+        plan = rk.rksc_plan_create_from_gate(batch.layout, batch.map_host.numpy(), batch.lists)
     else:
-        tables = batch.tables
-    plan = rk.rksc_plan_create(w.layout, tables)
+        plan = rk.rksc_plan_create(batch.layout, batch.tables)
     batch.ensure_buffers(plan)
     kw = dict(out=batch.out, block_mass=batch.mass, workspace=batch.workspace, device_status=batch.status)
     if seg_events is None:
@@ -223,7 +224,7 @@ def algorithmic_bytes(plan, layout):
     bpt = 2 * layout.num_kv_heads * layout.head_dim * 2
     kv = plan.unique_kv_tokens * bpt
     qb = plan.num_branches * layout.num_q_heads * layout.head_dim * 2
-    tables = 4 * int(plan.tables.seg_block_off[-1])
+    tables = 4 * plan.num_pages_listed
     mass = 4 * plan.mass_elems
     return kv, kv + qb + tables + mass
 
@@ -486,7 +487,7 @@ def punch_long_context(rk, batch: DeviceBatch):
     scores = sum(m[:, :npg].astype(np.float64).sum(axis=0) for m in masses)
     holed = workloads.punch_holes(w, 0, workloads.lowest_mass_pages(scores, 0.2))
     batch.w = holed
-    batch.tables = holed.tables
+    batch.tables = rk.Tables.of(holed.tables)
 
 
 def sweep_configs(rk, dev, flush, peak_gbs, skip, cached):

@@ -125,7 +125,10 @@ RKSC_API void rksc_tables_free(rksc_tables* t);
  * rksc_plan_create checks the tables (RKSC_ERR_BAD_TABLE), groups each segment with the
  * ascending list of branches that share it, cuts segments into KV chunks sized for the
  * device's SM count, lays out the partial-result workspace and the block-mass output, and
- * uploads its lists to the current device (synchronously; it may allocate device memory).
+ * uploads its lists to the current device (synchronously, on a stream of the library's own; device
+ * and pinned staging memory are taken from a small cache that destroyed plans return theirs to, so
+ * creating a plan per decode step does not allocate in the steady state).  A plan may be destroyed
+ * while its last launch is still running: its memory is not reused before that launch has finished.
  * Without a CUDA device the plan is host-only: it can be queried but not run.
  * A plan holds a small device-side work counter that a launch uses and rewinds, so a plan may
  * be in flight on one stream at a time (create one plan per concurrent stream).  It does not
@@ -142,9 +145,18 @@ typedef struct {
     int64_t unique_kv_tokens;    /* valid tokens of the distinct segments referenced       */
     int64_t duplicated_kv_tokens;/* sum over branches of the tokens they attend to        */
     int32_t on_device;           /* 1 when the lists were uploaded                        */
+    int64_t num_pages_listed;    /* page ids in the tables (sum of the segments' pages)    */
 } rksc_plan_info;
 
 RKSC_API int32_t rksc_plan_create(const rksc_layout* layout, const rksc_tables* tables, rksc_plan** out);
+/* rksc_tables_from_gate followed by rksc_plan_create, without handing the tables back: the usual
+ * per-step call when the tables come from the gate map (arguments as rksc_tables_from_gate). */
+RKSC_API int32_t rksc_plan_create_from_gate(const rksc_layout* layout, int32_t B, int32_t P,
+                              const int32_t* branch_to_prefix,
+                              const int32_t* shared_off, const int32_t* shared_pages, const int32_t* shared_ntok,
+                              const int32_t* priv_off,   const int32_t* priv_pages,   const int32_t* priv_ntok,
+                              const int32_t* sfx_off,    const int32_t* sfx_pages,    const int32_t* sfx_ntok,
+                              rksc_plan** out);
 RKSC_API int32_t rksc_plan_query(const rksc_plan* plan, rksc_plan_info* info);
 /* Work item i as 10 int32: segment, kv_head, first page (index within the segment), pages,
  * tokens, first sharer (index within the segment's sharer list), sharers, first partial row,

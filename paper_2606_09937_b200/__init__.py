@@ -17,6 +17,8 @@ from .binding import (  # noqa: F401
     rksc_asks_gate,
     rksc_tables_from_gate,
     rksc_plan_create,
+    rksc_plan_create_from_gate,
+    GateLists,
     rksc_branch_decode_attention,
     rksc_branch_decode_attention_static,
     rksc_decode_step_host,

@@ -23,6 +23,7 @@ EXPORTED_SYMBOLS = (
     "rksc_tables_from_gate",
     "rksc_tables_free",
     "rksc_plan_create",
+    "rksc_plan_create_from_gate",
     "rksc_plan_query",
     "rksc_plan_get_item",
     "rksc_plan_destroy",
@@ -59,7 +60,7 @@ class _CPlanInfo(C.Structure):
     _fields_ = [("workspace_bytes", C.c_size_t), ("mass_elems", C.c_int64),
                 ("mass_off", C.POINTER(C.c_int64)), ("num_work_items", C.c_int32),
                 ("num_partial_rows", C.c_int32), ("unique_kv_tokens", C.c_int64),
-                ("duplicated_kv_tokens", C.c_int64), ("on_device", C.c_int32)]
+                ("duplicated_kv_tokens", C.c_int64), ("on_device", C.c_int32), ("num_pages_listed", C.c_int64)]
 
 
 def lib_path() -> str:
@@ -90,6 +91,8 @@ def lib() -> C.CDLL:
     L.rksc_tables_free.argtypes = [C.POINTER(_CTables)]
     L.rksc_plan_create.restype = C.c_int32
     L.rksc_plan_create.argtypes = [C.POINTER(_CLayout), C.POINTER(_CTables), C.POINTER(C.c_void_p)]
+    L.rksc_plan_create_from_gate.restype = C.c_int32
+    L.rksc_plan_create_from_gate.argtypes = [C.POINTER(_CLayout), C.c_int32, C.c_int32] + [i32p] * 10 + [C.POINTER(C.c_void_p)]
     L.rksc_plan_query.restype = C.c_int32
     L.rksc_plan_query.argtypes = [C.c_void_p, C.POINTER(_CPlanInfo)]
     L.rksc_plan_get_item.restype = C.c_int32
@@ -199,22 +202,34 @@ def rksc_tables_from_gate(branch_to_prefix, num_prefixes,
 class Plan:
     """Owner of an rksc_plan (destroyed with the object)."""
 
-    def __init__(self, handle: int, layout: Layout, tables: Tables):
+    def __init__(self, handle: int, layout: Layout, tables: Optional[Tables], num_branches: int):
         self._h = C.c_void_p(handle)
         self.layout = layout
-        self.tables = tables
-        info = _CPlanInfo()
-        _check(lib().rksc_plan_query(self._h, C.byref(info)), "rksc_plan_query")
-        B = tables.c.num_branches
-        self.workspace_bytes = int(info.workspace_bytes)
-        self.mass_elems = int(info.mass_elems)
-        self.mass_off = np.ctypeslib.as_array(info.mass_off, shape=(B + 1,)).copy()
-        self.num_work_items = int(info.num_work_items)
-        self.num_partial_rows = int(info.num_partial_rows)
-        self.unique_kv_tokens = int(info.unique_kv_tokens)
-        self.duplicated_kv_tokens = int(info.duplicated_kv_tokens)
-        self.on_device = bool(info.on_device)
-        self.num_branches = B
+        self.tables = tables      # None when the plan was created straight from a gate map
+        self.num_branches = num_branches
+        self._info = None
+
+    def _query(self):
+        if self._info is None:
+            info = _CPlanInfo()
+            _check(lib().rksc_plan_query(self._h, C.byref(info)), "rksc_plan_query")
+            self._info = info
+            self._mass_off = np.ctypeslib.as_array(info.mass_off, shape=(self.num_branches + 1,)).copy()
+        return self._info
+
+    workspace_bytes = property(lambda self: int(self._query().workspace_bytes))
+    mass_elems = property(lambda self: int(self._query().mass_elems))
+    num_work_items = property(lambda self: int(self._query().num_work_items))
+    num_partial_rows = property(lambda self: int(self._query().num_partial_rows))
+    unique_kv_tokens = property(lambda self: int(self._query().unique_kv_tokens))
+    duplicated_kv_tokens = property(lambda self: int(self._query().duplicated_kv_tokens))
+    on_device = property(lambda self: bool(self._query().on_device))
+    num_pages_listed = property(lambda self: int(self._query().num_pages_listed))
+
+    @property
+    def mass_off(self):
+        self._query()
+        return self._mass_off
 
     def item(self, i: int) -> np.ndarray:
         out = np.zeros(10, dtype=np.int32)
@@ -242,7 +257,28 @@ def rksc_plan_create(layout, tables) -> Plan:
     tab = Tables.of(tables)
     h = C.c_void_p()
     _check(lib().rksc_plan_create(C.byref(lay.c), C.byref(tab.c), C.byref(h)), "rksc_plan_create")
-    return Plan(h.value, lay, tab)
+    return Plan(h.value, lay, tab, tab.c.num_branches)
+
+
+class GateLists:
+    """The nine CSR arrays of the two-level page lists, marshalled once and reusable across steps."""
+
+    def __init__(self, flat):
+        self.num_prefixes = int(flat.num_prefixes)
+        self.arrays = [_i32(getattr(flat, n)) for n in ("shared_off", "shared_pages", "shared_ntok", "priv_off",
+                                                       "priv_pages", "priv_ntok", "sfx_off", "sfx_pages", "sfx_ntok")]
+        self.ptrs = [_p(a) for a in self.arrays]
+
+
+def rksc_plan_create_from_gate(layout, branch_to_prefix, lists) -> Plan:
+    """rksc_tables_from_gate + rksc_plan_create in one host call (``lists``: a GateLists or an object with the CSR arrays)."""
+    lay = layout if isinstance(layout, Layout) else Layout.of(layout)
+    gl = lists if isinstance(lists, GateLists) else GateLists(lists)
+    m = _i32(branch_to_prefix)
+    h = C.c_void_p()
+    _check(lib().rksc_plan_create_from_gate(C.byref(lay.c), len(m), gl.num_prefixes, _p(m), *gl.ptrs, C.byref(h)),
+           "rksc_plan_create_from_gate")
+    return Plan(h.value, lay, None, len(m))
 
 
 def rksc_asks_gate(h_branch, h_root, cand_prefix, alpha: float, tau: float,

@@ -84,6 +84,73 @@ int32_t make_pool_map(const rksc_layout& L, const void* base, CUtensorMap* tm) {
     return r == CUDA_SUCCESS ? RKSC_OK : RKSC_ERR_CUDA;
 }
 
+// Device arenas (with a pinned staging buffer each) are recycled between plans: creating and
+// destroying a plan per decode step then costs no cudaMalloc / cudaFree.
+std::vector<PlanArena> g_arena_pool;            // guarded by g_mu
+cudaStream_t g_upload_stream[kMaxDevices];      // non-blocking: uploads do not wait for the caller's kernels
+
+int32_t acquire_arena(int dev, size_t bytes, PlanArena* out) {
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        int best = -1;
+        for (int i = 0; i < (int)g_arena_pool.size(); ++i)
+            if (g_arena_pool[i].device == dev && g_arena_pool[i].capacity >= bytes &&
+                (best < 0 || g_arena_pool[i].capacity < g_arena_pool[best].capacity))
+                best = i;
+        if (best >= 0) {
+            *out = g_arena_pool[best];
+            g_arena_pool.erase(g_arena_pool.begin() + best);
+        } else {
+            *out = PlanArena{};
+        }
+        if (!g_upload_stream[dev] &&
+            cudaStreamCreateWithFlags(&g_upload_stream[dev], cudaStreamNonBlocking) != cudaSuccess) {
+            cudaGetLastError();
+            return RKSC_ERR_CUDA;
+        }
+    }
+    if (out->dev) {
+        // the plan that used this arena last may still have work in flight
+        if (out->busy && cudaEventSynchronize(out->done) != cudaSuccess) cudaGetLastError();
+        out->busy = false;
+        return RKSC_OK;
+    }
+    size_t cap = 64 << 10;
+    while (cap < bytes) cap <<= 1;
+    PlanArena a{};
+    a.device = dev;
+    a.capacity = cap;
+    if (cudaMalloc(&a.dev, cap) != cudaSuccess || cudaMallocHost(&a.host, cap) != cudaSuccess ||
+        cudaEventCreateWithFlags(&a.done, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        if (a.dev) cudaFree(a.dev);
+        if (a.host) cudaFreeHost(a.host);
+        return RKSC_ERR_CUDA;
+    }
+    *out = a;
+    return RKSC_OK;
+}
+
+void release_arena(PlanArena a, bool used, cudaStream_t last_stream) {
+    if (!a.dev) return;
+    if (used) {
+        a.busy = (cudaEventRecord(a.done, last_stream) == cudaSuccess);
+        if (!a.busy) {
+            cudaGetLastError();
+            cudaStreamSynchronize(last_stream);
+        }
+    }
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (g_arena_pool.size() < 16) {
+        g_arena_pool.push_back(a);
+    } else {
+        if (a.busy) cudaEventSynchronize(a.done);
+        cudaFree(a.dev);
+        cudaFreeHost(a.host);
+        cudaEventDestroy(a.done);
+    }
+}
+
 template <typename T>
 size_t bytes_of(const std::vector<T>& v) {
     return (v.size() * sizeof(T) + 255) / 256 * 256;
@@ -98,12 +165,9 @@ int32_t upload_plan(rksc_plan* p) {
     size_t total = 0;
     for (size_t s : sizes) total += s;
     if (total == 0) total = 256;
-    std::vector<uint8_t> stage;
-    try {
-        stage.assign(total, 0);
-    } catch (const std::bad_alloc&) {
-        return RKSC_ERR_NOMEM;
-    }
+    int32_t st = acquire_arena(p->device, total, &p->arena);
+    if (st != RKSC_OK) return st;
+    uint8_t* stage = static_cast<uint8_t*>(p->arena.host);
     const void* srcs[kN] = {H.items.data(),      H.seg_blocks.data(), H.sharers.data(),      H.merge_off.data(),
                             H.merge_rows.data(), H.mass_off.data(),   H.br_nblk.data(),      nullptr};
     const size_t raw[kN] = {H.items.size() * sizeof(WorkItem), H.seg_blocks.size() * 4, H.sharers.size() * sizeof(Sharer),
@@ -112,21 +176,20 @@ int32_t upload_plan(rksc_plan* p) {
     size_t offs[kN], off = 0;
     for (int i = 0; i < kN; ++i) {
         offs[i] = off;
-        if (raw[i]) std::memcpy(stage.data() + off, srcs[i], raw[i]);
+        if (raw[i]) std::memcpy(stage + off, srcs[i], raw[i]);
+        else std::memset(stage + off, 0, sizes[i]);
         off += sizes[i];
     }
-    void* d = nullptr;
-    if (cudaMalloc(&d, total) != cudaSuccess) {
+    void* d = p->arena.dev;
+    cudaStream_t us = g_upload_stream[p->device];
+    if (cudaMemcpyAsync(d, stage, total, cudaMemcpyHostToDevice, us) != cudaSuccess ||
+        cudaStreamSynchronize(us) != cudaSuccess) {
         cudaGetLastError();
-        return RKSC_ERR_CUDA;
-    }
-    if (cudaMemcpy(d, stage.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) {
-        cudaGetLastError();
-        cudaFree(d);
+        release_arena(p->arena, false, nullptr);
+        p->arena = PlanArena{};
         return RKSC_ERR_CUDA;
     }
     uint8_t* base = static_cast<uint8_t*>(d);
-    p->dev_arena = d;
     p->dev.items = reinterpret_cast<const WorkItem*>(base + offs[0]);
     p->dev.seg_blocks = reinterpret_cast<const int32_t*>(base + offs[1]);
     p->dev.sharers = reinterpret_cast<const Sharer*>(base + offs[2]);
@@ -210,6 +273,22 @@ extern "C" RKSC_API int32_t rksc_plan_create(const rksc_layout* layout, const rk
     return RKSC_OK;
 }
 
+extern "C" RKSC_API int32_t rksc_plan_create_from_gate(
+    const rksc_layout* layout, int32_t B, int32_t P, const int32_t* branch_to_prefix, const int32_t* shared_off,
+    const int32_t* shared_pages, const int32_t* shared_ntok, const int32_t* priv_off, const int32_t* priv_pages,
+    const int32_t* priv_ntok, const int32_t* sfx_off, const int32_t* sfx_pages, const int32_t* sfx_ntok,
+    rksc_plan** out) {
+    if (!out) return RKSC_ERR_INVALID_ARG;
+    *out = nullptr;
+    rksc_tables t;
+    int32_t st = rksc_tables_from_gate(B, P, branch_to_prefix, shared_off, shared_pages, shared_ntok, priv_off,
+                                       priv_pages, priv_ntok, sfx_off, sfx_pages, sfx_ntok, &t);
+    if (st != RKSC_OK) return st;
+    st = rksc_plan_create(layout, &t, out);
+    rksc_tables_free(&t);
+    return st;
+}
+
 extern "C" RKSC_API int32_t rksc_plan_query(const rksc_plan* plan, rksc_plan_info* info) {
     if (!plan || !info) return RKSC_ERR_INVALID_ARG;
     const HostPlan& H = plan->host;
@@ -221,6 +300,7 @@ extern "C" RKSC_API int32_t rksc_plan_query(const rksc_plan* plan, rksc_plan_inf
     info->unique_kv_tokens = H.unique_kv_tokens;
     info->duplicated_kv_tokens = H.duplicated_kv_tokens;
     info->on_device = plan->on_device ? 1 : 0;
+    info->num_pages_listed = (int64_t)H.seg_blocks.size();
     return RKSC_OK;
 }
 
@@ -244,11 +324,11 @@ extern "C" RKSC_API int32_t rksc_plan_get_item(const rksc_plan* plan, int32_t i,
 
 extern "C" RKSC_API void rksc_plan_destroy(rksc_plan* plan) {
     if (!plan) return;
-    if (plan->dev_arena) {
+    if (plan->arena.dev) {
         int cur = -1;
         const bool sw = (cudaGetDevice(&cur) == cudaSuccess && cur != plan->device && plan->device >= 0);
         if (sw) cudaSetDevice(plan->device);
-        cudaFree(plan->dev_arena);
+        release_arena(plan->arena, plan->used, static_cast<cudaStream_t>(plan->last_stream));
         if (sw) cudaSetDevice(cur);
     }
     delete plan;
@@ -309,6 +389,8 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
     a.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    plan->used = true;
+    plan->last_stream = stream;
     cudaError_t e = cudaSuccess;
     if (phases & RKSC_PHASE_SEGMENTS) {
         e = launch_seg_attn_tc(tm_k, tm_v, a, s);

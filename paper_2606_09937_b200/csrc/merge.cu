@@ -8,8 +8,10 @@
 //   mass_j = 2^(logmass_j - LSE)
 // which is exactly softmax attention over the concatenation of the branch's segments.
 //
-// One warp per (branch, head): lanes split the head dimension four columns each (16-byte loads of
-// the partial rows) and stride over the parts and the blocks.  The kernel is launched with
+// One warp (or, when there are few (branch, head) pairs, 2/4/8 warps) per (branch, head): lanes split
+// the head dimension four columns each (16-byte loads of the partial rows) and stride over the parts;
+// the warps of a pair each recompute the (cheap) LSE and share out the pair's blocks, so that the
+// mass pass has enough loads in flight even when B x Hq is small and the context is long.  The kernel is launched with
 // programmatic stream serialisation: its blocks may become resident while the segment kernel
 // drains, read their (plan-owned) part lists, and then wait for the segment kernel's results.
 #include "kernels.h"
@@ -28,9 +30,11 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 
 __global__ void __launch_bounds__(kMergeThreads)
-merge_kernel(const AttnArgs a) {
+merge_kernel(const AttnArgs a, const int wpk_log2) {
     const int lane = threadIdx.x & 31;
-    const int bh = blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
+    const int gw = blockIdx.x * kMergeWarps + (threadIdx.x >> 5);   // global warp
+    const int bh = gw >> wpk_log2;
+    const int sub = gw & ((1 << wpk_log2) - 1), wpk = 1 << wpk_log2;
     const bool live = bh < a.B * a.Hq;
     int b = 0, h = 0, lo = 0, hi = 0;
     if (live) {
@@ -66,10 +70,10 @@ merge_kernel(const AttnArgs a) {
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     const float lse = mx + log2f(sum);
 
-    // out: lane owns columns 4*lane .. 4*lane+3
+    // out (first warp of the pair): lane owns columns 4*lane .. 4*lane+3
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    const bool has_cols = 4 * lane < HD;
-    for (int i0 = lo; i0 < hi; i0 += 32) {
+    const bool has_cols = (4 * lane < HD) && sub == 0;
+    for (int i0 = lo; i0 < hi && sub == 0; i0 += 32) {
         const int n = min(32, hi - i0);
         const int my_row = (i0 == lo) ? row_l : ((i0 + lane < hi) ? a.plan.merge_rows[i0 + lane] + gi : -1);
         const float my_w = (my_row >= 0) ? fast_exp2(a.part_lse[my_row] - lse) : 0.f;
@@ -90,7 +94,16 @@ merge_kernel(const AttnArgs a) {
     if (a.block_mass != nullptr && hi > lo) {
         const int nblk = a.plan.br_nblk[b];
         float* mass = a.block_mass + a.plan.mass_off[b] * a.Hq + (int64_t)h * nblk;
-        for (int j = lane; j < nblk; j += 32) mass[j] = fast_exp2(mass[j] - lse);
+        const int stride = 32 * wpk;
+        int j = sub * 32 + lane;
+        for (; j + 3 * stride < nblk; j += 4 * stride) {   // four independent loads in flight
+            const float v0 = mass[j], v1 = mass[j + stride], v2 = mass[j + 2 * stride], v3 = mass[j + 3 * stride];
+            mass[j] = fast_exp2(v0 - lse);
+            mass[j + stride] = fast_exp2(v1 - lse);
+            mass[j + 2 * stride] = fast_exp2(v2 - lse);
+            mass[j + 3 * stride] = fast_exp2(v3 - lse);
+        }
+        for (; j < nblk; j += stride) mass[j] = fast_exp2(mass[j] - lse);
     }
 }
 
@@ -99,8 +112,11 @@ merge_kernel(const AttnArgs a) {
 cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream) {
     const int n = a.B * a.Hq;
     if (n == 0) return cudaSuccess;
+    int wpk_log2 = 0;   // warps per (branch, head): enough warps to fill the device
+    while (wpk_log2 < 3 && ((int64_t)n << (wpk_log2 + 1)) <= 8192) ++wpk_log2;
+    const int64_t warps = (int64_t)n << wpk_log2;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((n + kMergeWarps - 1) / kMergeWarps, 1, 1);
+    cfg.gridDim = dim3((unsigned)((warps + kMergeWarps - 1) / kMergeWarps), 1, 1);
     cfg.blockDim = dim3(kMergeThreads, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
@@ -109,7 +125,7 @@ cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, merge_kernel, a);
+    return cudaLaunchKernelEx(&cfg, merge_kernel, a, wpk_log2);
 }
 
 }  // namespace rksc

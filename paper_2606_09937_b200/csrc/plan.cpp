@@ -135,6 +135,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     const int base = (int)std::min<int64_t>(128, std::max<int64_t>(kMinChunk, fair / 6));
 
     int64_t rows_total = 0;
+    P.items.reserve((size_t)(total_units / std::max(1, std::min(cap, base)) + 2 * (int64_t)S * L.num_kv_heads));
     for (int s = 0; s < S; ++s) {
         const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
         const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
@@ -173,10 +174,18 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
 
     // tensor-core items first, then warp-MMA items; within a class longest first, so that the
     // CTAs, which claim items in this order, finish together
-    std::stable_sort(P.items.begin(), P.items.end(), [G](const WorkItem& a, const WorkItem& b) {
-        if (a.klass != b.klass) return a.klass > b.klass;
-        return item_cost(a, G) > item_cost(b, G);
-    });
+    {
+        const size_t n = P.items.size();
+        std::vector<uint64_t> keys(n);
+        for (size_t i = 0; i < n; ++i) {
+            const uint64_t cost = (uint64_t)item_cost(P.items[i], G);               // < 2^24
+            keys[i] = ((uint64_t)(1 - P.items[i].klass) << 56) | ((((uint64_t)1 << 24) - 1 - cost) << 32) | (uint64_t)i;
+        }
+        std::sort(keys.begin(), keys.end());   // class 1 first, then descending cost, then creation order
+        std::vector<WorkItem> sorted(n);
+        for (size_t i = 0; i < n; ++i) sorted[i] = P.items[(uint32_t)keys[i]];
+        P.items.swap(sorted);
+    }
     int32_t row = 0;
     P.num_tc_items = 0;
     for (auto& it : P.items) {
@@ -235,8 +244,11 @@ extern "C" RKSC_API int32_t rksc_tables_from_gate(int32_t B, int32_t P, const in
     std::vector<int32_t> shared_seg(P > 0 ? P : 1, -1);
     std::vector<int32_t> seg_off{0}, blocks, ntok, br_segs((size_t)2 * B);
     try {
+        seg_off.reserve((size_t)P + 2 * (size_t)B + 1);
+        ntok.reserve((size_t)P + 2 * (size_t)B);
+        blocks.reserve((size_t)(P > 0 ? shared_off[P] : 0) + (size_t)(B > 0 ? priv_off[B] + sfx_off[B] : 0));
         auto add = [&](const int32_t* off, const int32_t* pages, const int32_t* nt, int i) {
-            for (int k = off[i]; k < off[i + 1]; ++k) blocks.push_back(pages[k]);
+            if (off[i + 1] > off[i]) blocks.insert(blocks.end(), pages + off[i], pages + off[i + 1]);
             seg_off.push_back((int32_t)blocks.size());
             ntok.push_back(nt[i]);
             return (int32_t)ntok.size() - 1;

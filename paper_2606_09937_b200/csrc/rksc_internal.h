@@ -81,10 +81,24 @@ int32_t build_host_plan(const rksc_layout& layout, const rksc_tables& t, int num
 
 }  // namespace rksc
 
+namespace rksc {
+// Device memory of a plan's lists, with the pinned buffer they are staged in; recycled between plans.
+struct PlanArena {
+    void* dev = nullptr;
+    void* host = nullptr;          // pinned
+    size_t capacity = 0;
+    int device = -1;
+    struct CUevent_st* done = nullptr;   // cudaEvent_t, recorded when a plan that ran is destroyed
+    bool busy = false;
+};
+}  // namespace rksc
+
 struct rksc_plan {
     rksc::HostPlan host;
     rksc::DevicePlan dev;
-    void* dev_arena = nullptr;
+    rksc::PlanArena arena;
+    mutable bool used = false;          // a launch was enqueued with this plan
+    mutable void* last_stream = nullptr;
     int device = -1;
     int num_sms = 148;
     bool on_device = false;
