@@ -35,7 +35,7 @@ FALLBACK_HBM_GBS = 6650.0    # used only when MEASURED_PEAKS.json is absent
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the segment kernel, from the ncu
 # capture summarised under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"batched_serving": 777373952}   # profiles/seg_attention_batched_serving.md
 
 WORKLOAD_LABEL = {
     "tiny": "configs[0] tiny: 8q/2kv d64, 4 branches, prefix 256 + suffix 32",
@@ -60,6 +60,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-config attention-only table")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-pipeline", action="store_true", help="time the steps strictly one after another")
     return ap.parse_args()
 
 
@@ -201,6 +202,59 @@ def run_step(rk, batch: DeviceBatch, seg_events=None):
         rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=2, **kw)
     launches += 2
     return plan, launches
+
+
+class StepContext:
+    """Per-step buffers and stream for the software-pipelined loop (two steps in flight)."""
+
+    def __init__(self, batch: DeviceBatch, plan):
+        import torch
+        dev = batch.dev
+        B = batch.q.shape[0]
+        self.stream = torch.cuda.Stream(device=dev)
+        self.map_dev = torch.empty(B, dtype=torch.int32, device=dev)
+        self.sigma_dev = torch.empty(B, dtype=torch.float32, device=dev)
+        self.map_host = torch.empty(B, dtype=torch.int32).pin_memory()
+        self.ev_map = torch.cuda.Event()
+        self.out = torch.empty_like(batch.out)
+        self.mass = torch.empty_like(batch.mass)
+        self.workspace = torch.empty_like(batch.workspace)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.plan = None
+
+
+def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events):
+    """K steps with two in flight: while the attention of step i runs on one stream, the gate of step
+    i+1 runs on the other and the host builds step i+1's plan from its map.  Every step still does the
+    whole path (gate kernel, map to the host, tables + plan, segment kernels, merge).  Returns launches."""
+    import torch
+    w = batch.w
+    g = w.gate
+
+    def gate_stage(ctx):
+        rk.rksc_asks_gate(batch.h_branch, batch.h_root, batch.cand, g.alpha, g.tau,
+                          branch_to_prefix=ctx.map_dev, sigma=ctx.sigma_dev, stream=ctx.stream)
+        with torch.cuda.stream(ctx.stream):
+            ctx.map_host.copy_(ctx.map_dev, non_blocking=True)
+        ctx.ev_map.record(ctx.stream)
+
+    def attention_stage(ctx, ev):
+        ctx.ev_map.synchronize()                       # the host needs the map to build the tables
+        plan = rk.rksc_plan_create_from_gate(batch.layout, ctx.map_host.numpy(), batch.lists)
+        kw = dict(out=ctx.out, block_mass=ctx.mass, workspace=ctx.workspace, device_status=ctx.status,
+                  stream=ctx.stream)
+        ev[0].record(ctx.stream)
+        rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=1, **kw)
+        ev[1].record(ctx.stream)
+        rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=2, **kw)
+        ctx.plan = plan                                # the previous plan of this context is released here
+
+    gate_stage(ctxs[0])
+    for i in range(steps):
+        if i + 1 < steps:
+            gate_stage(ctxs[(i + 1) % 2])
+        attention_stage(ctxs[i % 2], seg_events[i])
+    return 3 * steps
 
 
 def attention_only_times(rk, batch: DeviceBatch, plan, iters: int, flush):
@@ -354,11 +408,39 @@ def run_ours(args):
         launches += n
     barrier()
     t_wall = time.perf_counter() - t_wall0
-    clocks = sampler.stop() if rank == 0 else None
     step_ms = [a.elapsed_time(b) for a, b in step_ev]
     seg_ms = [a.elapsed_time(b) for a, b in seg_ev]
     total_ms = sum(step_ms)           # device time of exactly K steps (flushes excluded)
     assert int(batch.status.item()) == 0, "a kernel reported a device-side timeout"
+    serial = {"ms_per_step": total_ms / args.steps, "wall_ms_per_step": t_wall * 1e3 / args.steps,
+              "tbps_unique_kv": kv_bytes * args.steps / (total_ms * 1e-3) / 1e12,
+              "what": "the same K steps strictly one after another on one stream"}
+    pipelined = batch.has_gate and not small and not args.no_pipeline
+    if pipelined:
+        # the headline loop: two steps in flight on two streams (see pipelined_steps)
+        ctxs = [StepContext(batch, plan), StepContext(batch, plan)]
+        warm_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(4)]
+        pipelined_steps(rk, batch, ctxs, 4, warm_ev)
+        torch.cuda.synchronize()
+        seg_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                  for _ in range(args.steps)]
+        e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t_wall0 = time.perf_counter()
+        e_start.record()
+        for c in ctxs:
+            c.stream.wait_event(e_start)
+        launches = pipelined_steps(rk, batch, ctxs, args.steps, seg_ev)
+        for c in ctxs:
+            torch.cuda.current_stream().wait_stream(c.stream)
+        e_end.record()
+        barrier()
+        t_wall = time.perf_counter() - t_wall0
+        total_ms = e_start.elapsed_time(e_end)
+        seg_ms = [a.elapsed_time(b) for a, b in seg_ev]
+        for c in ctxs:
+            assert int(c.status.item()) == 0, "a kernel reported a device-side timeout"
+    clocks = sampler.stop() if rank == 0 else None
     value, total_ms_max = aggregate_over_ranks(dist, dev, kv_bytes, args.steps, total_ms)
     peak_gbs, peak_kind = measured_peak_gbs()
     seg_avg_ms = sum(seg_ms) / len(seg_ms)
@@ -371,7 +453,9 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
             "workload": WORKLOAD_LABEL[args.workload],
-            "step": "gate kernel + map D2H + tables + plan + attention (segment kernel + merge)",
+            "step": "gate kernel + map D2H + tables + plan + attention (segment kernels + merge)",
+            "pipelining": ("two steps in flight on two streams: the gate of step i+1 runs and its plan is built on the "
+                           "host while the attention of step i runs") if pipelined else "none (steps strictly serial)",
             "unique_kv_bytes": kv_bytes, "branches": B, "work_items": plan.num_work_items,
             "l2": ("inputs larger than L2 (unique KV %.0f MB vs L2 %.0f MB)" % (kv_bytes / 1e6, l2_bytes / 1e6))
             if not small else "L2 flushed (write of 2x L2) before every timed step",
@@ -382,6 +466,7 @@ def run_ours(args):
         "pct_of_measured_copy_peak": 100.0 * value * 1e3 / world / peak_gbs,
         "wall_ms_per_step": t_wall * 1e3 / args.steps,
         "gpu_launches": launches,
+        "serial_steps": serial,
         "roofline": {
             "kernel": "segment attention: seg_attn_tc_kernel + seg_attn_warp_kernel (chained launches)", "bound": "hbm", "achieved": achieved, "peak": peak_gbs,
             "unit": "GB/s", "frac": achieved / peak_gbs, "peak_source": peak_kind,

@@ -130,11 +130,16 @@ def _p(a: np.ndarray):
     return a.ctypes.data_as(C.POINTER(C.c_int32))
 
 
-def _stream_ptr(stream) -> int:
+def _stream_ptr(stream, device=None) -> int:
+    """Raw cudaStream_t of ``stream`` (a torch stream), or of torch's current stream on ``device``."""
     import torch
-    if stream is None:
-        stream = torch.cuda.current_stream()
-    return int(stream.cuda_stream)
+    if stream is not None:
+        return int(stream.cuda_stream)
+    idx = device.index if (device is not None and device.index is not None) else torch.cuda.current_device()
+    try:
+        return int(torch._C._cuda_getCurrentRawStream(idx))   # cheap; the public call re-probes the driver
+    except AttributeError:
+        return int(torch.cuda.current_stream(idx).cuda_stream)
 
 
 class Layout:
@@ -297,7 +302,7 @@ def rksc_asks_gate(h_branch, h_root, cand_prefix, alpha: float, tau: float,
         sigma = torch.empty(B, dtype=torch.float32, device=h_branch.device)
     st = lib().rksc_asks_gate(h_branch.data_ptr(), h_root.data_ptr(), cand_prefix.data_ptr(), B, P, L, D,
                               float(alpha), float(tau), branch_to_prefix.data_ptr(), sigma.data_ptr(),
-                              _stream_ptr(stream))
+                              _stream_ptr(stream, h_branch.device))
     _check(st, "rksc_asks_gate")
     return branch_to_prefix, sigma
 
@@ -328,7 +333,7 @@ def rksc_branch_decode_attention(plan: Plan, q, k_pool, v_pool, out=None, block_
     args = (plan._h, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), out.data_ptr(),
             block_mass.data_ptr() if block_mass is not None else None,
             workspace.data_ptr(), workspace.numel() * workspace.element_size(),
-            device_status.data_ptr(), _stream_ptr(stream))
+            device_status.data_ptr(), _stream_ptr(stream, dev))
     if phases == 3:
         st = lib().rksc_branch_decode_attention(*args)
     else:
@@ -358,7 +363,7 @@ def rksc_branch_decode_attention_static(plan: Plan, q, k_pool, v_pool, out, bloc
     st = lib().rksc_branch_decode_attention_static(
         plan._h, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), out.data_ptr(),
         block_mass.data_ptr() if block_mass is not None else None,
-        device_status.data_ptr() if device_status is not None else None, _stream_ptr(stream))
+        device_status.data_ptr() if device_status is not None else None, _stream_ptr(stream, q.device))
     _check(st, "rksc_branch_decode_attention_static")
     return out, block_mass, device_status
 
@@ -386,6 +391,6 @@ def rksc_decode_step_host(layout, h_branch, h_root, cand_prefix, alpha, tau, fla
         *[_p(a) for a in lists], q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(),
         branch_to_prefix.data_ptr(), sigma.data_ptr() if sigma is not None else None, out.data_ptr(),
         block_mass.data_ptr() if block_mass is not None else None,
-        block_mass.numel() if block_mass is not None else 0, mo, _stream_ptr(stream))
+        block_mass.numel() if block_mass is not None else 0, mo, _stream_ptr(stream, k_pool.device))
     _check(st, "rksc_decode_step_host")
     return st
