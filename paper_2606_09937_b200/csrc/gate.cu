@@ -1,6 +1,6 @@
 // ASKS similarity gate (paper Eq. 2, Algorithm 2) as one launch.
 //
-// One thread-block cluster per branch.  Every warp of the cluster takes whole layers: it
+// One thread-block cluster (up to 4 CTAs of 8 warps) per branch.  Every warp of the cluster takes whole layers: it
 // streams the branch's and the candidate root's D-vector of that layer once with 16-byte
 // loads, reduces dot / |h_b|^2 / |h_r|^2 with warp shuffles, and accumulates
 // exp(alpha*(l-L)/L) * cos_l and exp(alpha*(l-L)/L) (the factor exp(-alpha) cancels in the
@@ -18,9 +18,9 @@ namespace rksc {
 
 namespace {
 
-constexpr int kGateWarps = 4;
+constexpr int kGateWarps = 8;
 constexpr int kGateThreads = kGateWarps * 32;
-constexpr int kMaxCluster = 8;
+constexpr int kMaxCluster = 4;
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -135,7 +135,8 @@ asks_gate_kernel(const float* __restrict__ h_branch, const float* __restrict__ h
 cudaError_t launch_asks_gate(const float* h_branch, const float* h_root, const int32_t* cand_prefix,
                              int B, int P, int L, int D, float alpha, float tau,
                              int32_t* branch_to_prefix, float* sigma, cudaStream_t stream) {
-    // cluster size: enough warps to give every layer its own warp, at most 8 CTAs
+    // cluster size: enough warps to give every layer its own warp, at most kMaxCluster CTAs (larger
+    // clusters of smaller CTAs were measured to limit how many clusters the device keeps resident)
     int csize = 1;
     while (csize < kMaxCluster && csize * kGateWarps < L) csize <<= 1;
     const bool vec4 = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(h_branch) & 15) == 0) &&
