@@ -223,13 +223,16 @@ class StepContext:
         self.plan = None
 
 
-def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events):
-    """K steps with two in flight: while the attention of step i runs on one stream, the gate of step
-    i+1 runs on the other and the host builds step i+1's plan from its map.  Every step still does the
-    whole path (gate kernel, map to the host, tables + plan, segment kernels, merge).  Returns launches."""
+def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events, pool):
+    """K steps, software-pipelined three deep over len(ctxs) = 3 contexts (stream + buffers each):
+    while the attention of step i runs, the gate kernel of step i+2 is already enqueued and a host
+    worker thread builds step i+1's plan from its map (the C calls release the interpreter lock).
+    Every step still does the whole path: gate kernel, map to the host, tables + plan, segment
+    kernels, merge.  Returns the number of kernel launches."""
     import torch
     w = batch.w
     g = w.gate
+    n = len(ctxs)
 
     def gate_stage(ctx):
         rk.rksc_asks_gate(batch.h_branch, batch.h_root, batch.cand, g.alpha, g.tau,
@@ -238,22 +241,32 @@ def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events):
             ctx.map_host.copy_(ctx.map_dev, non_blocking=True)
         ctx.ev_map.record(ctx.stream)
 
-    def attention_stage(ctx, ev):
+    def plan_stage(ctx):
         ctx.ev_map.synchronize()                       # the host needs the map to build the tables
-        plan = rk.rksc_plan_create_from_gate(batch.layout, ctx.map_host.numpy(), batch.lists)
+        return rk.rksc_plan_create_from_gate(batch.layout, ctx.map_host.numpy(), batch.lists)
+
+    def attention_stage(ctx, plan, ev):
         kw = dict(out=ctx.out, block_mass=ctx.mass, workspace=ctx.workspace, device_status=ctx.status,
                   stream=ctx.stream)
-        ev[0].record(ctx.stream)
-        rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=1, **kw)
-        ev[1].record(ctx.stream)
-        rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=2, **kw)
-        ctx.plan = plan                                # the previous plan of this context is released here
+        if ev is None:
+            rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, **kw)
+        else:                                          # every few steps: events around the segment kernels
+            ev[0].record(ctx.stream)
+            rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=1, **kw)
+            ev[1].record(ctx.stream)
+            rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=2, **kw)
+        ctx.plan = plan                                # the context's previous plan is released here
 
     gate_stage(ctxs[0])
+    if steps > 1:
+        gate_stage(ctxs[1 % n])
+    fut = pool.submit(plan_stage, ctxs[0])
     for i in range(steps):
-        if i + 1 < steps:
-            gate_stage(ctxs[(i + 1) % 2])
-        attention_stage(ctxs[i % 2], seg_events[i])
+        if i + 2 < steps:
+            gate_stage(ctxs[(i + 2) % n])
+        nxt = pool.submit(plan_stage, ctxs[(i + 1) % n]) if i + 1 < steps else None
+        attention_stage(ctxs[i % n], fut.result(), seg_events.get(i))
+        fut = nxt
     return 3 * steps
 
 
@@ -418,26 +431,29 @@ def run_ours(args):
     pipelined = batch.has_gate and not small and not args.no_pipeline
     if pipelined:
         # the headline loop: two steps in flight on two streams (see pipelined_steps)
-        ctxs = [StepContext(batch, plan), StepContext(batch, plan)]
-        warm_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(4)]
-        pipelined_steps(rk, batch, ctxs, 4, warm_ev)
+        from concurrent.futures import ThreadPoolExecutor
+        pool = ThreadPoolExecutor(max_workers=1)
+        ctxs = [StepContext(batch, plan) for _ in range(3)]
+        pipelined_steps(rk, batch, ctxs, 6, {}, pool)
         torch.cuda.synchronize()
-        seg_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                  for _ in range(args.steps)]
+        # events around the segment kernels on every 4th step (they cost two extra host calls)
+        seg_ev = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                  for i in range(0, args.steps, 4)}
         e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         t_wall0 = time.perf_counter()
         e_start.record()
         for c in ctxs:
             c.stream.wait_event(e_start)
-        launches = pipelined_steps(rk, batch, ctxs, args.steps, seg_ev)
+        launches = pipelined_steps(rk, batch, ctxs, args.steps, seg_ev, pool)
         for c in ctxs:
             torch.cuda.current_stream().wait_stream(c.stream)
         e_end.record()
         barrier()
         t_wall = time.perf_counter() - t_wall0
+        pool.shutdown()
         total_ms = e_start.elapsed_time(e_end)
-        seg_ms = [a.elapsed_time(b) for a, b in seg_ev]
+        seg_ms = [a.elapsed_time(b) for a, b in seg_ev.values()]
         for c in ctxs:
             assert int(c.status.item()) == 0, "a kernel reported a device-side timeout"
     clocks = sampler.stop() if rank == 0 else None
@@ -454,8 +470,9 @@ def run_ours(args):
         "config": {
             "workload": WORKLOAD_LABEL[args.workload],
             "step": "gate kernel + map D2H + tables + plan + attention (segment kernels + merge)",
-            "pipelining": ("two steps in flight on two streams: the gate of step i+1 runs and its plan is built on the "
-                           "host while the attention of step i runs") if pipelined else "none (steps strictly serial)",
+            "pipelining": ("three steps in flight (3 streams): while the attention of step i runs, the gate of step "
+                           "i+2 is enqueued and a host thread builds the plan of step i+1") if pipelined
+            else "none (steps strictly serial)",
             "unique_kv_bytes": kv_bytes, "branches": B, "work_items": plan.num_work_items,
             "l2": ("inputs larger than L2 (unique KV %.0f MB vs L2 %.0f MB)" % (kv_bytes / 1e6, l2_bytes / 1e6))
             if not small else "L2 flushed (write of 2x L2) before every timed step",

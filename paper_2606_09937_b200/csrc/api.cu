@@ -87,6 +87,7 @@ int32_t make_pool_map(const rksc_layout& L, const void* base, CUtensorMap* tm) {
 // Device arenas (with a pinned staging buffer each) are recycled between plans: creating and
 // destroying a plan per decode step then costs no cudaMalloc / cudaFree.
 std::vector<PlanArena> g_arena_pool;            // guarded by g_mu
+std::vector<rksc_plan*> g_plan_pool;            // destroyed plan objects, kept for their vectors' capacity
 cudaStream_t g_upload_stream[kMaxDevices];      // non-blocking: uploads do not wait for the caller's kernels
 
 int32_t acquire_arena(int dev, size_t bytes, PlanArena* out) {
@@ -243,8 +244,23 @@ extern "C" RKSC_API const char* rksc_last_cuda_error(void) { return cudaGetError
 extern "C" RKSC_API int32_t rksc_plan_create(const rksc_layout* layout, const rksc_tables* tables, rksc_plan** out) {
     if (!layout || !tables || !out) return RKSC_ERR_INVALID_ARG;
     *out = nullptr;
-    rksc_plan* p = new (std::nothrow) rksc_plan();
+    rksc_plan* p = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_plan_pool.empty()) {
+            p = g_plan_pool.back();
+            g_plan_pool.pop_back();
+        }
+    }
+    if (!p) p = new (std::nothrow) rksc_plan();
     if (!p) return RKSC_ERR_NOMEM;
+    p->dev = DevicePlan{};
+    p->arena = PlanArena{};
+    p->used = false;
+    p->last_stream = nullptr;
+    p->device = -1;
+    p->num_sms = 148;
+    p->on_device = false;
     int ndev = 0;
     const bool have_dev = (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0);
     if (!have_dev) cudaGetLastError();
@@ -330,6 +346,13 @@ extern "C" RKSC_API void rksc_plan_destroy(rksc_plan* plan) {
         if (sw) cudaSetDevice(plan->device);
         release_arena(plan->arena, plan->used, static_cast<cudaStream_t>(plan->last_stream));
         if (sw) cudaSetDevice(cur);
+    }
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (g_plan_pool.size() < 8) {
+            g_plan_pool.push_back(plan);
+            return;
+        }
     }
     delete plan;
 }

@@ -63,7 +63,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
         if (t.br_segs[i] < 0 || t.br_segs[i] >= S) return RKSC_ERR_BAD_TABLE;
 
     HostPlan& P = *hp;
-    P = HostPlan{};
+    P.reset();
     P.layout = L;
     P.B = B;
     P.S = S;
@@ -95,7 +95,8 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     for (int s = 0; s < S; ++s) P.seg_sharer_off[s + 1] += P.seg_sharer_off[s];
     P.sharers.resize(total_refs);
     {
-        std::vector<int32_t> fill(P.seg_sharer_off.begin(), P.seg_sharer_off.end() - 1);
+        std::vector<int32_t>& fill = P.scratch_a;
+        fill.assign(P.seg_sharer_off.begin(), P.seg_sharer_off.end() - 1);
         for (int b = 0; b < B; ++b) {
             int64_t loff = 0;
             for (int i = t.br_seg_off[b]; i < t.br_seg_off[b + 1]; ++i) {
@@ -135,7 +136,20 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     const int base = (int)std::min<int64_t>(128, std::max<int64_t>(kMinChunk, fair / 6));
 
     int64_t rows_total = 0;
-    P.items.reserve((size_t)(total_units / std::max(1, std::min(cap, base)) + 2 * (int64_t)S * L.num_kv_heads));
+    {
+        size_t n_items = 0;   // exact count, so that the item vector is allocated once
+        for (int s = 0; s < S; ++s) {
+            const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
+            const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
+            if (ns == 0 || np == 0) continue;
+            const int nsb = ceil_div(ns, seg_rows_per_block(ns));
+            for (int sb = 0; sb < nsb; ++sb) {
+                const int rows = ((int)((int64_t)ns * (sb + 1) / nsb) - (int)((int64_t)ns * sb / nsb)) * G;
+                n_items += (size_t)ceil_div(np, std::min(cap, std::max(base, 2 * rows))) * L.num_kv_heads;
+            }
+        }
+        P.items.reserve(n_items);
+    }
     for (int s = 0; s < S; ++s) {
         const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
         const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
@@ -175,15 +189,30 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     // tensor-core items first, then warp-MMA items; within a class longest first, so that the
     // CTAs, which claim items in this order, finish together
     {
+        // counting sort on (class, cost / 16): descending cost up to the bucket width is all the
+        // longest-first claiming needs, and it is linear in the number of items
         const size_t n = P.items.size();
-        std::vector<uint64_t> keys(n);
+        constexpr int kBuckets = 1024;
+        std::vector<int32_t>& bucket_of = P.scratch_a;
+        bucket_of.resize(n);
+        int32_t count[2][kBuckets + 1];
+        std::memset(count, 0, sizeof(count));
         for (size_t i = 0; i < n; ++i) {
-            const uint64_t cost = (uint64_t)item_cost(P.items[i], G);               // < 2^24
-            keys[i] = ((uint64_t)(1 - P.items[i].klass) << 56) | ((((uint64_t)1 << 24) - 1 - cost) << 32) | (uint64_t)i;
+            const int64_t cost = item_cost(P.items[i], G);
+            const int bkt = kBuckets - 1 - (int)std::min<int64_t>(kBuckets - 1, cost >> 4);   // small index = long item
+            bucket_of[i] = bkt;
+            count[1 - P.items[i].klass][bkt + 1]++;
         }
-        std::sort(keys.begin(), keys.end());   // class 1 first, then descending cost, then creation order
-        std::vector<WorkItem> sorted(n);
-        for (size_t i = 0; i < n; ++i) sorted[i] = P.items[(uint32_t)keys[i]];
+        int32_t start[2][kBuckets];
+        int32_t run = 0;
+        for (int c = 0; c < 2; ++c)
+            for (int b = 0; b < kBuckets; ++b) {
+                start[c][b] = run;
+                run += count[c][b + 1];
+            }
+        std::vector<WorkItem>& sorted = P.scratch_items;
+        sorted.resize(n);
+        for (size_t i = 0; i < n; ++i) sorted[start[1 - P.items[i].klass][bucket_of[i]]++] = P.items[i];
         P.items.swap(sorted);
     }
     int32_t row = 0;
@@ -206,7 +235,8 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     for (int k = 0; k < nkeys; ++k) P.merge_off[k + 1] += P.merge_off[k];
     P.merge_rows.resize(P.merge_off[nkeys]);
     {
-        std::vector<int32_t> fill(P.merge_off.begin(), P.merge_off.end() - 1);
+        std::vector<int32_t>& fill = P.scratch_b;
+        fill.assign(P.merge_off.begin(), P.merge_off.end() - 1);
         for (const auto& it : P.items)
             for (int i = 0; i < it.num_sharers; ++i) {
                 const int key = P.sharers[it.sharer_begin + i].branch * L.num_kv_heads + it.kv_head;

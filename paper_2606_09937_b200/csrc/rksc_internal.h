@@ -74,6 +74,31 @@ struct HostPlan {
     int64_t unique_kv_tokens = 0, duplicated_kv_tokens = 0;
     size_t workspace_bytes = 0;
     size_t ws_lse_offset = 0;             // byte offset of the lse array inside the workspace
+    // scratch of build_host_plan, kept so that a recycled plan object allocates nothing
+    std::vector<WorkItem> scratch_items;
+    std::vector<int32_t> scratch_a, scratch_b;
+
+    // Back to an empty plan; the vectors keep their capacity.
+    void reset() {
+        layout = rksc_layout{};
+        B = S = 0;
+        G = 1;
+        seg_blocks.clear();
+        seg_block_off.clear();
+        seg_num_tokens.clear();
+        items.clear();
+        num_tc_items = grid_tc = grid_warp = 0;
+        sharers.clear();
+        seg_sharer_off.clear();
+        merge_off.clear();
+        merge_rows.clear();
+        mass_off.clear();
+        br_nblk.clear();
+        mass_elems = 0;
+        num_partial_rows = 0;
+        unique_kv_tokens = duplicated_kv_tokens = 0;
+        workspace_bytes = ws_lse_offset = 0;
+    }
 };
 
 // Builds every host list from validated tables.  num_sms sizes the KV chunks.
