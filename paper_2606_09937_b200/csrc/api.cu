@@ -70,17 +70,13 @@ int32_t get_encode(EncodeTiledFn* fn) {
 
 // The pool viewed as a 2-D bf16 tensor [num_pool_blocks * Hkv * 16 rows][head_dim], fetched in
 // boxes of 16 rows x 64 columns (128 bytes) with the 128-byte swizzle.
-// `whole_tile`: the same memory viewed as rows of 64 elements ([... * head_dim/64 rows][64]) and fetched
-// in boxes of one whole (page, kv head) tile, 16 * head_dim/64 rows.
-int32_t make_pool_map(const rksc_layout& L, const void* base, CUtensorMap* tm, bool whole_tile = false) {
+int32_t make_pool_map(const rksc_layout& L, const void* base, CUtensorMap* tm) {
     EncodeTiledFn enc;
     int32_t st = get_encode(&enc);
     if (st != RKSC_OK) return st;
-    const cuuint64_t rows = (cuuint64_t)L.num_pool_blocks * L.num_kv_heads * kBlock;
-    const cuuint32_t halves = (cuuint32_t)(L.head_dim / 64);
-    const cuuint64_t gdim[2] = {whole_tile ? 64u : (cuuint64_t)L.head_dim, whole_tile ? rows * halves : rows};
-    const cuuint64_t gstride[1] = {whole_tile ? 128u : (cuuint64_t)L.head_dim * 2};
-    const cuuint32_t box[2] = {64, whole_tile ? (cuuint32_t)kBlock * halves : (cuuint32_t)kBlock};
+    const cuuint64_t gdim[2] = {(cuuint64_t)L.head_dim, (cuuint64_t)L.num_pool_blocks * L.num_kv_heads * kBlock};
+    const cuuint64_t gstride[1] = {(cuuint64_t)L.head_dim * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kBlock};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -393,11 +389,6 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
     if (st != RKSC_OK) return st;
     st = make_pool_map(H.layout, v_pool, &tm_v);
     if (st != RKSC_OK) return st;
-    CUtensorMap tm_k_tile, tm_v_tile;   // whole-tile boxes, for the warp-per-item kernel
-    st = make_pool_map(H.layout, k_pool, &tm_k_tile, true);
-    if (st != RKSC_OK) return st;
-    st = make_pool_map(H.layout, v_pool, &tm_v_tile, true);
-    if (st != RKSC_OK) return st;
 
     AttnArgs a{};
     a.plan = plan->dev;
@@ -410,10 +401,8 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
     a.counters = plan->dev.counters;
     a.num_items = (int)H.items.size();
     a.num_tc_items = H.num_tc_items;
-    a.num_small_items = H.num_small_items;
     a.grid_warp = H.grid_warp;
     a.grid_tc = H.grid_tc;
-    a.grid_small = H.grid_small;
     a.B = H.B;
     a.Hq = H.layout.num_q_heads;
     a.Hkv = H.layout.num_kv_heads;
@@ -427,12 +416,8 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
     plan->last_stream = stream;
     cudaError_t e = cudaSuccess;
     if (phases & RKSC_PHASE_SEGMENTS) {
-        // tensor-core items, then single-warp items, then cooperative-warp items; each later kernel is
-        // launched to start as the earlier one drains and does not complete before it has
         e = launch_seg_attn_tc(tm_k, tm_v, a, s);
-        if (e == cudaSuccess) e = launch_seg_attn_small(tm_k_tile, tm_v_tile, a, s, /*chained=*/a.grid_tc > 0);
-        if (e == cudaSuccess)
-            e = launch_seg_attn_warp(tm_k, tm_v, a, s, /*chained=*/a.grid_tc > 0 || a.grid_small > 0);
+        if (e == cudaSuccess) e = launch_seg_attn_warp(tm_k, tm_v, a, s, /*after_tc=*/a.grid_tc > 0);
     }
     if (e == cudaSuccess && (phases & RKSC_PHASE_MERGE)) e = launch_merge(a, s);
     if (e != cudaSuccess) {

@@ -212,7 +212,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         // at a time one batch ahead, so that no global-memory latency sits between two TMA issues.
         auto claim = [&]() {   // this kernel's items follow the tcgen05 kernel's in the item array
             int v = 0;
-            if (lane == 0) v = a.num_tc_items + a.num_small_items + atomicAdd(a.counters, 1);
+            if (lane == 0) v = a.num_tc_items + atomicAdd(a.counters, 1);
             return __shfl_sync(0xffffffffu, v, 0);
         };
         auto fetch_item = [&](int i) {
@@ -714,12 +714,9 @@ size_t warp_kernel_smem_bytes(int head_dim) {
 }
 
 cudaError_t configure_tc_kernel();
-cudaError_t configure_small_kernel();
 
 cudaError_t configure_attention_kernels() {
     cudaError_t e = configure_tc_kernel();
-    if (e != cudaSuccess) return e;
-    e = configure_small_kernel();
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(seg_attn_warp_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)warp_kernel_smem_bytes(128));

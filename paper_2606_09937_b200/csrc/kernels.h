@@ -22,9 +22,8 @@ struct AttnArgs {
     int32_t* status;        // may be null
     int32_t* counters;      // [2]: next work item, CTAs done; zero between launches
     int num_items;
-    int num_tc_items;       // items [0, num_tc_items) go to the tcgen05 kernel,
-    int num_small_items;    // the next num_small_items to the warp-per-item kernel, the rest to the cooperative warp kernel
-    int grid_warp, grid_tc, grid_small;   // persistent CTAs of the three segment kernels
+    int num_tc_items;       // items [0, num_tc_items) go to the tcgen05 kernel, the rest to the warp kernel
+    int grid_warp, grid_tc; // persistent CTAs of the two segment kernels
     int B, Hq, Hkv, G, head_dim;
     float scale_log2;       // sm_scale * log2(e)
 };
@@ -39,10 +38,6 @@ size_t tc_kernel_smem_bytes();
 // starts as that one drains (programmatic dependent launch) and waits for it before it exits.
 cudaError_t launch_seg_attn_warp(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnArgs& a,
                                  cudaStream_t stream, bool after_tc);
-// chained: another segment kernel was launched just before on the stream (as for the warp kernel)
-cudaError_t launch_seg_attn_small(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnArgs& a,
-                                  cudaStream_t stream, bool chained);
-size_t small_kernel_smem_bytes(int head_dim);
 cudaError_t launch_seg_attn_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnArgs& a,
                                cudaStream_t stream);
 cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream);

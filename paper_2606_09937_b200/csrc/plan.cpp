@@ -113,8 +113,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
 
     // Work items.  A segment whose stacked rows (sharers x G) reach kTcMinRows goes to the
     // tensor-core (tcgen05) kernel in sharer blocks of up to 128 rows; the rest goes to the
-    // warp-MMA kernels in blocks of up to 64 rows: blocks of at most 8 rows to the kernel whose
-    // warps work alone, the others to the kernel whose warps share pages.  KV chunks are long enough that the partial
+    // warp-MMA kernel in blocks of up to 64 rows.  KV chunks are long enough that the partial
     // results stay a few percent of the KV bytes read (their size grows with the stacked rows)
     // and short enough that the persistent CTAs end together.
     const bool tc_ok = (L.head_dim == 128) && !env_flag("RKSC_DISABLE_TC");
@@ -132,27 +131,10 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     }
     const int max_grid = std::max(1, num_sms) * kCtasPerSm;
     const int kMinChunk = 8;
-    // Small-row blocks go to the warp-per-item kernel only when there is enough of them to give every
-    // warp of the device several items' worth of pages; a small problem is latency-bound and does better
-    // with four warps sharing an item (the cooperative kernel).
-    int64_t small_units = 0;
-    for (int s = 0; s < S; ++s) {
-        const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
-        const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
-        if (ns * G <= kSmallMaxRows && ns > 0) small_units += (int64_t)np * L.num_kv_heads;
-    }
-    const bool small_ok = !env_flag("RKSC_DISABLE_SMALL") &&
-                          small_units >= (int64_t)max_grid * kSmallWarpsPerCta * 2 * kSmallMaxPages;
     const int64_t fair = total_units / max_grid;                     // page-heads per CTA
     const int cap = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, fair * 2 / 3));
     const int base = (int)std::min<int64_t>(128, std::max<int64_t>(kMinChunk, fair / 6));
 
-    // pages per chunk: small-row items are processed by single warps that hold an item's page ids in
-    // one register per lane, hence at most 32 pages
-    auto chunk_pages = [&](int rows, int klass) {
-        const int want = std::min(cap, std::max(base, 2 * rows));
-        return klass == 2 ? std::min(want, kSmallMaxPages) : want;
-    };
     int64_t rows_total = 0;
     {
         size_t n_items = 0;   // exact count, so that the item vector is allocated once
@@ -163,8 +145,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
             const int nsb = ceil_div(ns, seg_rows_per_block(ns));
             for (int sb = 0; sb < nsb; ++sb) {
                 const int rows = ((int)((int64_t)ns * (sb + 1) / nsb) - (int)((int64_t)ns * sb / nsb)) * G;
-                const int klass = (tc_ok && rows >= kTcMinRows) ? 1 : ((small_ok && rows <= kSmallMaxRows) ? 2 : 0);
-                n_items += (size_t)ceil_div(np, chunk_pages(rows, klass)) * L.num_kv_heads;
+                n_items += (size_t)ceil_div(np, std::min(cap, std::max(base, 2 * rows))) * L.num_kv_heads;
             }
         }
         P.items.reserve(n_items);
@@ -178,8 +159,8 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
             // balanced split of the sharers
             const int sh_lo = (int)((int64_t)ns * sb / nsb), sh_hi = (int)((int64_t)ns * (sb + 1) / nsb);
             const int rows = (sh_hi - sh_lo) * G;
-            const int klass = (tc_ok && rows >= kTcMinRows) ? 1 : ((small_ok && rows <= kSmallMaxRows) ? 2 : 0);
-            const int want = chunk_pages(rows, klass);
+            const int klass = (tc_ok && rows >= kTcMinRows) ? 1 : 0;
+            const int want = std::min(cap, std::max(base, 2 * rows));
             const int nch = ceil_div(np, want);
             for (int c = 0; c < nch; ++c) {
                 const int p_lo = (int)((int64_t)np * c / nch), p_hi = (int)((int64_t)np * (c + 1) / nch);
@@ -214,39 +195,36 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
         constexpr int kBuckets = 1024;
         std::vector<int32_t>& bucket_of = P.scratch_a;
         bucket_of.resize(n);
-        int32_t count[3][kBuckets + 1];
+        int32_t count[2][kBuckets + 1];
         std::memset(count, 0, sizeof(count));
-        auto rank_of = [](int klass) { return klass == 1 ? 0 : (klass == 2 ? 1 : 2); };   // launch order of the kernels
         for (size_t i = 0; i < n; ++i) {
             const int64_t cost = item_cost(P.items[i], G);
             const int bkt = kBuckets - 1 - (int)std::min<int64_t>(kBuckets - 1, cost >> 4);   // small index = long item
             bucket_of[i] = bkt;
-            count[rank_of(P.items[i].klass)][bkt + 1]++;
+            count[1 - P.items[i].klass][bkt + 1]++;
         }
-        int32_t start[3][kBuckets];
+        int32_t start[2][kBuckets];
         int32_t run = 0;
-        for (int c = 0; c < 3; ++c)
+        for (int c = 0; c < 2; ++c)
             for (int b = 0; b < kBuckets; ++b) {
                 start[c][b] = run;
                 run += count[c][b + 1];
             }
         std::vector<WorkItem>& sorted = P.scratch_items;
         sorted.resize(n);
-        for (size_t i = 0; i < n; ++i) sorted[start[rank_of(P.items[i].klass)][bucket_of[i]]++] = P.items[i];
+        for (size_t i = 0; i < n; ++i) sorted[start[1 - P.items[i].klass][bucket_of[i]]++] = P.items[i];
         P.items.swap(sorted);
     }
     int32_t row = 0;
-    P.num_tc_items = P.num_small_items = 0;
+    P.num_tc_items = 0;
     for (auto& it : P.items) {
         it.part_row_base = row;
         row += it.num_sharers * G;
-        P.num_tc_items += (it.klass == 1);
-        P.num_small_items += (it.klass == 2);
+        P.num_tc_items += it.klass;
     }
     P.num_partial_rows = row;
     P.grid_tc = std::min(std::max(1, num_sms), P.num_tc_items);
-    P.grid_small = std::min(max_grid, ceil_div(P.num_small_items, kSmallWarpsPerCta));
-    P.grid_warp = std::min(max_grid, (int)P.items.size() - P.num_tc_items - P.num_small_items);
+    P.grid_warp = std::min(max_grid, (int)P.items.size() - P.num_tc_items);
 
     // merge lists: for every (branch, kv head) the partial rows (of head-in-group 0) to combine
     const int nkeys = B * L.num_kv_heads;

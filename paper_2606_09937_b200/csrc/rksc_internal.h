@@ -13,9 +13,6 @@ constexpr int kBlock = RKSC_BLOCK_SIZE;     // tokens per KV page
 constexpr int kMaxRowsPerItem = 64;         // stacked query rows one warp-MMA work item handles
 constexpr int kTcMinRows = 17;              // from this many stacked rows on, the tcgen05 kernel takes the item
 constexpr int kTcMaxRows = 128;             // rows of one tcgen05 work item (the MMA's M)
-constexpr int kSmallMaxRows = 8;            // up to this many rows an item goes to the warp-per-item kernel
-constexpr int kSmallMaxPages = 32;          // pages of such an item (one page id per lane)
-constexpr int kSmallWarpsPerCta = 4;
 constexpr int kMaxPagesPerItem = 512;       // page ids a CTA caches in shared memory
 constexpr int kConsumerWarps = 4;           // MMA warps of the segment kernel
 constexpr int kWarpKernelThreads = (kConsumerWarps + 1) * 32;   // + one TMA producer warp
@@ -35,7 +32,7 @@ struct WorkItem {
     int32_t num_sharers;
     int32_t part_row_base;   // first row of this item's partial results
     int32_t seg_page_begin;  // index of the first page within its segment
-    int32_t klass;           // 0: cooperative warp-MMA kernel, 1: tcgen05 kernel, 2: warp-per-item kernel
+    int32_t klass;           // 0: warp-MMA kernel, 1: tcgen05 kernel
 };
 static_assert(sizeof(WorkItem) == 40, "WorkItem is read as 10 int32");
 
@@ -54,7 +51,7 @@ struct DevicePlan {
     const int32_t* merge_rows = nullptr;  // partial row of head-in-group 0 for each part
     const int64_t* mass_off = nullptr;    // [B+1]
     const int32_t* br_nblk = nullptr;     // [B]
-    int32_t* counters = nullptr;          // [6] work-claim counters (cooperative warp kernel, tcgen05 kernel, warp-per-item kernel), zero between launches
+    int32_t* counters = nullptr;          // [4] work-claim counters (warp kernel, tcgen05 kernel), zero between launches
 };
 
 struct HostPlan {
@@ -64,9 +61,8 @@ struct HostPlan {
     std::vector<int32_t> seg_block_off;
     std::vector<int32_t> seg_num_tokens;
     std::vector<WorkItem> items;
-    int32_t num_tc_items = 0;             // items [0, num_tc_items) belong to the tcgen05 kernel,
-    int32_t num_small_items = 0;          // the next num_small_items to the warp-per-item kernel, the rest to the cooperative one
-    int32_t grid_tc = 0, grid_small = 0, grid_warp = 0;   // persistent CTAs of the three segment kernels
+    int32_t num_tc_items = 0;             // items [0, num_tc_items) belong to the tcgen05 kernel
+    int32_t grid_tc = 0, grid_warp = 0;   // persistent CTAs of the two segment kernels
     std::vector<Sharer> sharers;
     std::vector<int32_t> seg_sharer_off;  // [S+1]
     std::vector<int32_t> merge_off;
@@ -91,7 +87,7 @@ struct HostPlan {
         seg_block_off.clear();
         seg_num_tokens.clear();
         items.clear();
-        num_tc_items = num_small_items = grid_tc = grid_small = grid_warp = 0;
+        num_tc_items = grid_tc = grid_warp = 0;
         sharers.clear();
         seg_sharer_off.clear();
         merge_off.clear();

@@ -52,12 +52,8 @@ def test_plan_covers_every_page_row_pair_once(maker):
     for seg, kvh, p0, npg, ntok, s0, ns, prow, klass, _ in items.tolist():
         assert npg >= 1 and ns >= 1
         assert ns * G <= (128 if klass == 1 else 64)
-        if klass == 1:      # tensor-core kernel
+        if klass == 1:
             assert ns * G >= 17 and L.head_dim == 128
-        elif klass == 2:    # warp-per-item kernel
-            assert ns * G <= 8 and npg <= 32
-        else:               # cooperative warp kernel (also takes small rows when the problem is small)
-            assert ns * G <= 64
         seg_pages = int(t.seg_block_off[seg + 1] - t.seg_block_off[seg])
         assert p0 + npg <= seg_pages and s0 + ns <= len(sharers[seg])
         assert ntok == min(int(t.seg_num_tokens[seg]), (p0 + npg) * 16) - p0 * 16
@@ -80,16 +76,6 @@ def test_plan_covers_every_page_row_pair_once(maker):
     assert p.unique_kv_tokens * L.bytes_per_token == workloads.unique_kv_bytes(L, t)
     assert p.duplicated_kv_tokens * L.bytes_per_token == workloads.duplicated_kv_bytes(L, t)
     assert p.workspace_bytes >= p.num_partial_rows * (L.head_dim + 1) * 4
-
-
-def test_small_rows_go_to_the_warp_per_item_kernel_only_in_large_problems():
-    # few pages: four warps share an item (class 0)
-    w = workloads.make_from_segments("few", 16, 8, 64, [300] * 8, [[b] for b in range(8)], seed=4)
-    assert set(_plan_for(w).items()[:, 8].tolist()) == {0}
-    # many pages of 2-row items: every warp works alone on items of at most 32 pages (class 2)
-    w = workloads.make_from_segments("many", 16, 8, 64, [1216] * 128, [[b] for b in range(128)], seed=4)
-    items = _plan_for(w).items()
-    assert set(items[:, 8].tolist()) == {2} and items[:, 3].max() <= 32
 
 
 def test_plan_rejects_bad_tables_and_layouts():
