@@ -508,11 +508,16 @@ def run_ours(args):
         if not args.no_sweep:
             line["configs"] = sweep_configs(rk, dev, flush, peak_gbs, skip=args.workload, cached=(args.workload, line))
         if not args.no_cpu_baseline:
-            dt, ub, cores, nb, Bt = oracle_pass(w, args.cpu_sample_branches)
+            # about 10-30 s of oracle work: whole passes over the batch until 10 s have gone by
+            passes, total, ub, cores, nb, Bt = 0, 0.0, 0, 1, 0, 0
+            while total < 10.0 and passes < 8:
+                dt, ub, cores, nb, Bt = oracle_pass(w, args.cpu_sample_branches)
+                total += dt
+                passes += 1
             line["cpu_baseline"] = {
-                "value": ub / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "value": ub * passes / total / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
                 "sample": f"{nb} of {Bt} branches of the batch (gate over all branches, attention over these), "
-                          f"one pass, {dt:.1f} s", "seconds": dt}
+                          f"{passes} passes, {total:.1f} s in all", "seconds": total}
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
