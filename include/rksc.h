@@ -75,6 +75,9 @@ RKSC_API int32_t rksc_asks_gate(const float* h_branch, const float* h_root, cons
  *
  * Pool: K and V are separate dev tensors [num_pool_blocks][num_kv_heads][16][head_dim] bf16,
  * 16-byte aligned.  Query head h reads KV head h / (num_q_heads / num_kv_heads).
+ * Token slots of a listed page that lie past its segment's token count are never attended to
+ * (their scores are masked and their probabilities are exactly 0), but they are fetched with the
+ * page and multiplied by those zeros: they must hold finite values (not NaN / Inf).
  *
  * Tables (segment form): segment s owns pages seg_blocks[seg_block_off[s] .. seg_block_off[s+1])
  * and seg_num_tokens[s] tokens; every page but the last is full, the last holds at least one
