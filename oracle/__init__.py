@@ -16,6 +16,8 @@ written for reading rather than speed:
                          prefix + suffix (the paper's repeat_interleave + clone,
                          Section 2.2 "KV broadcast and batched decode"), plus the
                          softmax mass per KV block.
+* ``page_scores`` / ``rsbcm_evict`` - the eviction that consumes those masses
+                         (Section 2.4, Algorithm 4).
 
 Parity pins: every function here is pinned by the CPU tests against closed
 forms, brute force on tiny inputs and invariants; none is "parity unpinned".
@@ -28,3 +30,4 @@ from .block_tables import (  # noqa: F401
     mass_offsets,
 )
 from .branch_attention import branch_decode_attention, to_f32_numpy  # noqa: F401
+from .rsbcm import page_scores, rsbcm_evict  # noqa: F401
