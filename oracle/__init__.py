@@ -30,4 +30,4 @@ from .block_tables import (  # noqa: F401
     mass_offsets,
 )
 from .branch_attention import branch_decode_attention, to_f32_numpy  # noqa: F401
-from .rsbcm import page_scores, rsbcm_evict  # noqa: F401
+from .rsbcm import page_scores, rsbcm_evict, apply_eviction  # noqa: F401

@@ -68,3 +68,26 @@ def test_page_scores_sum_and_sharing():
     sc2 = oracle.page_scores(w2.tables.seg_block_off, w2.tables.br_seg_off, w2.tables.br_segs, m2, 8)
     lo, hi = int(w2.tables.seg_block_off[1]), int(w2.tables.seg_block_off[2])     # the unused private copy
     assert np.all(sc2[lo:hi] == 0) and abs(sc2.sum() - 4 * 8) < 1e-10
+
+
+def test_apply_eviction_hand_case_and_hole_puncher():
+    # one segment of 3 pages holding 40 tokens (16 + 16 + 8), one of 1 page holding 5
+    off, blocks, ntok = np.array([0, 3, 4]), np.array([7, 3, 9, 2]), np.array([40, 5])
+    o, b, n = oracle.apply_eviction(off, blocks, ntok, np.array([0, 1, 0, 0], bool))
+    assert o.tolist() == [0, 2, 3] and b.tolist() == [7, 9, 2] and n.tolist() == [24, 5]
+    o, b, n = oracle.apply_eviction(off, blocks, ntok, np.array([0, 0, 1, 1], bool))      # partial tail pages go
+    assert o.tolist() == [0, 2, 2] and b.tolist() == [7, 3] and n.tolist() == [32, 0]
+    o, b, n = oracle.apply_eviction(off, blocks, ntok, np.zeros(4, bool))
+    assert o.tolist() == off.tolist() and b.tolist() == blocks.tolist() and n.tolist() == ntok.tolist()
+    # against the workload generator's hole puncher, one segment at a time
+    w = workloads.make_tiny()
+    t = w.tables
+    rng = np.random.default_rng(3)
+    ev = rng.random(int(t.seg_block_off[-1])) < 0.4
+    o, b, n = oracle.apply_eviction(t.seg_block_off, t.seg_blocks, t.seg_num_tokens, ev)
+    w2 = w
+    for s in range(len(t.seg_num_tokens)):
+        lo, hi = int(t.seg_block_off[s]), int(t.seg_block_off[s + 1])
+        w2 = workloads.punch_holes(w2, s, np.flatnonzero(ev[lo:hi]))
+    assert o.tolist() == w2.tables.seg_block_off.tolist() and b.tolist() == w2.tables.seg_blocks.tolist()
+    assert n.tolist() == w2.tables.seg_num_tokens.tolist()
