@@ -266,6 +266,55 @@ RKSC_API int32_t rksc_branch_decode_attention_static(const rksc_plan* plan, cons
                                      float* out, float* block_mass,
                                      int32_t* device_status, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * RSBCM eviction (paper Section 2.4 "RSBCM" and Algorithm 4), fed by the attention's block
+ * masses.  The paper ranks a cached block by omega = score / (depth + 1) and, while more than
+ * N_max blocks are cached, evicts the block with the smallest omega.  It does not say how an
+ * attention-derived score is formed; here the score of a table entry e = seg_block_off[s] + p
+ * (page p of segment s) is the softmax mass that every (branch, query head) attending to the
+ * segment put on that page, summed.
+ *
+ * rksc_rsbcm_page_scores: score[e] for every entry the plan's tables list (device, fp64,
+ * [num_pages_listed]).  score[e] = sum over the branches b listing s, in ascending b (a branch
+ * listing s twice counts twice), of (sum over heads h = 0..Hq-1 of block_mass[b][h][j]), j the
+ * logical block of the page in b.  Each head sum is formed first, in ascending h, then added to
+ * the running score, all in fp64 and in exactly this order: the result is defined bit for bit.
+ * block_mass is the array rksc_branch_decode_attention wrote for the same plan.
+ * Errors: RKSC_ERR_INVALID_ARG (NULL argument, plan without device lists), RKSC_ERR_CUDA.
+ * ------------------------------------------------------------------------------------------ */
+RKSC_API int32_t rksc_rsbcm_page_scores(const rksc_plan* plan, const float* block_mass, double* score,
+                                        void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * rksc_rsbcm_evict: Algorithm 4 on n entries.  omega[i] = score[i] / (depth[i] + 1) as one IEEE
+ * fp64 division; with k = max(0, n - capacity) the k entries that are smallest by (omega, i)
+ * are marked - the set the paper's loop (evict the arg-min, the first of equal minima, until at
+ * most N_max = capacity entries remain) ends with, since evicting an entry changes no other
+ * entry's omega.
+ *
+ * Device arguments: score fp64 [n] (finite), depth int32 [n] (>= 0), evicted uint8 [n] (out,
+ * 1 = evict, every element written), num_evicted int32 [1] (out, may be NULL), workspace of at
+ * least rksc_rsbcm_workspace_bytes(n) bytes, 256-byte aligned, contents irrelevant before and
+ * undefined after.  The selection runs in one thread block (an exact radix select over the
+ * 64 bits of omega), so its time grows linearly with n.
+ * Errors: RKSC_ERR_INVALID_ARG (NULL argument, n < 0, n >= 2^31), RKSC_ERR_WORKSPACE, RKSC_ERR_CUDA.
+ * ------------------------------------------------------------------------------------------ */
+RKSC_API size_t rksc_rsbcm_workspace_bytes(int64_t n);
+RKSC_API int32_t rksc_rsbcm_evict(const double* score, const int32_t* depth, int64_t n, int64_t capacity,
+                                  uint8_t* evicted, int32_t* num_evicted, void* workspace,
+                                  size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * rksc_tables_drop_evicted: the tables after eviction (host arrays in, host arrays out).  Each
+ * segment keeps its surviving pages in order; a dropped page takes its tokens with it (every
+ * page of a segment holds RKSC_BLOCK_SIZE tokens except the last, which holds the remainder); a
+ * segment may end up empty.  Branch lists are copied unchanged.  evicted is uint8
+ * [seg_block_off[S]].  `out` is allocated by the library: release it with rksc_tables_free.
+ * Errors: RKSC_ERR_INVALID_ARG, RKSC_ERR_BAD_TABLE (offsets not ascending, token count that
+ * does not fit the page count), RKSC_ERR_NOMEM.
+ * ------------------------------------------------------------------------------------------ */
+RKSC_API int32_t rksc_tables_drop_evicted(const rksc_tables* in, const uint8_t* evicted, rksc_tables* out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,6 +22,10 @@ from .binding import (  # noqa: F401
     rksc_branch_decode_attention,
     rksc_branch_decode_attention_static,
     rksc_decode_step_host,
+    rksc_rsbcm_page_scores,
+    rksc_rsbcm_workspace_bytes,
+    rksc_rsbcm_evict,
+    rksc_tables_drop_evicted,
     STATIC_WORKSPACE_BYTES,
     split_block_mass,
     EXPORTED_SYMBOLS,

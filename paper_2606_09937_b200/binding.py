@@ -31,6 +31,10 @@ EXPORTED_SYMBOLS = (
     "rksc_branch_decode_attention_phases",
     "rksc_branch_decode_attention_static",
     "rksc_decode_step_host",
+    "rksc_rsbcm_page_scores",
+    "rksc_rsbcm_workspace_bytes",
+    "rksc_rsbcm_evict",
+    "rksc_tables_drop_evicted",
 )
 STATIC_WORKSPACE_BYTES = 16 << 20
 
@@ -109,6 +113,15 @@ def lib() -> C.CDLL:
                                         [C.c_int64, C.c_void_p, C.c_void_p])
     L.rksc_branch_decode_attention_static.restype = C.c_int32
     L.rksc_branch_decode_attention_static.argtypes = [C.c_void_p] * 8
+    L.rksc_rsbcm_page_scores.restype = C.c_int32
+    L.rksc_rsbcm_page_scores.argtypes = [C.c_void_p] * 4
+    L.rksc_rsbcm_workspace_bytes.restype = C.c_size_t
+    L.rksc_rsbcm_workspace_bytes.argtypes = [C.c_int64]
+    L.rksc_rsbcm_evict.restype = C.c_int32
+    L.rksc_rsbcm_evict.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                   C.c_size_t, C.c_void_p]
+    L.rksc_tables_drop_evicted.restype = C.c_int32
+    L.rksc_tables_drop_evicted.argtypes = [C.POINTER(_CTables), C.c_void_p, C.POINTER(_CTables)]
     _lib = L
     return L
 
@@ -366,6 +379,60 @@ def rksc_branch_decode_attention_static(plan: Plan, q, k_pool, v_pool, out, bloc
         device_status.data_ptr() if device_status is not None else None, _stream_ptr(stream, q.device))
     _check(st, "rksc_branch_decode_attention_static")
     return out, block_mass, device_status
+
+
+def rksc_rsbcm_page_scores(plan: Plan, block_mass, score=None, stream=None):
+    """RSBCM score of every table entry (Section 2.4): device fp64 [num_pages_listed] from the block
+    masses the attention wrote for ``plan``."""
+    import torch
+    if score is None:
+        score = torch.empty(plan.num_pages_listed, dtype=torch.float64, device=block_mass.device)
+    st = lib().rksc_rsbcm_page_scores(plan._h, block_mass.data_ptr(), score.data_ptr(),
+                                      _stream_ptr(stream, block_mass.device))
+    _check(st, "rksc_rsbcm_page_scores")
+    return score
+
+
+def rksc_rsbcm_workspace_bytes(n: int) -> int:
+    return int(lib().rksc_rsbcm_workspace_bytes(int(n)))
+
+
+def rksc_rsbcm_evict(score, depth, capacity: int, evicted=None, num_evicted=None, workspace=None, stream=None):
+    """Algorithm 4 on device arrays: marks the max(0, n - capacity) entries smallest by
+    (score / (depth + 1), index).  Returns (evicted uint8 [n], num_evicted int32 [1])."""
+    import torch
+    n = int(score.numel())
+    dev = score.device
+    if evicted is None:
+        evicted = torch.empty(n, dtype=torch.uint8, device=dev)
+    if num_evicted is None:
+        num_evicted = torch.empty(1, dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(rksc_rsbcm_workspace_bytes(n), dtype=torch.uint8, device=dev)
+    st = lib().rksc_rsbcm_evict(score.data_ptr(), depth.data_ptr(), n, int(capacity), evicted.data_ptr(),
+                                num_evicted.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                _stream_ptr(stream, dev))
+    _check(st, "rksc_rsbcm_evict")
+    return evicted, num_evicted
+
+
+def rksc_tables_drop_evicted(tables, evicted) -> Tables:
+    """Host call: the tables without the evicted entries (``evicted``: host uint8/bool [entries])."""
+    t = Tables.of(tables)
+    ev = np.ascontiguousarray(np.asarray(evicted).astype(np.uint8))
+    out = _CTables()
+    st = lib().rksc_tables_drop_evicted(C.byref(t.c), ev.ctypes.data_as(C.c_void_p), C.byref(out))
+    _check(st, "rksc_tables_drop_evicted")
+    try:
+        S, B = out.num_segments, out.num_branches
+        cp = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(max(n, 1),))[:n].copy()
+        seg_block_off = cp(out.seg_block_off, S + 1)
+        br_seg_off = cp(out.br_seg_off, B + 1)
+        res = Tables(seg_block_off, cp(out.seg_blocks, int(seg_block_off[-1])), cp(out.seg_num_tokens, S),
+                     br_seg_off, cp(out.br_segs, int(br_seg_off[-1])))
+    finally:
+        lib().rksc_tables_free(C.byref(out))
+    return res
 
 
 def rksc_decode_step_host(layout, h_branch, h_root, cand_prefix, alpha, tau, flat, q, k_pool, v_pool,

@@ -159,10 +159,11 @@ size_t bytes_of(const std::vector<T>& v) {
 
 int32_t upload_plan(rksc_plan* p) {
     HostPlan& H = p->host;
-    constexpr int kN = 8;
+    constexpr int kN = 11;
     const size_t sizes[kN] = {bytes_of(H.items),      bytes_of(H.seg_blocks), bytes_of(H.sharers),
                               bytes_of(H.merge_off),  bytes_of(H.merge_rows), bytes_of(H.mass_off),
-                              bytes_of(H.br_nblk),    256 /* counters, zeroed */};
+                              bytes_of(H.br_nblk),    256 /* counters, zeroed */,
+                              bytes_of(H.seg_block_off), bytes_of(H.seg_sharer_off), bytes_of(H.score_chunks)};
     size_t total = 0;
     for (size_t s : sizes) total += s;
     if (total == 0) total = 256;
@@ -170,10 +171,13 @@ int32_t upload_plan(rksc_plan* p) {
     if (st != RKSC_OK) return st;
     uint8_t* stage = static_cast<uint8_t*>(p->arena.host);
     const void* srcs[kN] = {H.items.data(),      H.seg_blocks.data(), H.sharers.data(),      H.merge_off.data(),
-                            H.merge_rows.data(), H.mass_off.data(),   H.br_nblk.data(),      nullptr};
+                            H.merge_rows.data(), H.mass_off.data(),   H.br_nblk.data(),      nullptr,
+                            H.seg_block_off.data(), H.seg_sharer_off.data(), H.score_chunks.data()};
     const size_t raw[kN] = {H.items.size() * sizeof(WorkItem), H.seg_blocks.size() * 4, H.sharers.size() * sizeof(Sharer),
                             H.merge_off.size() * 4,            H.merge_rows.size() * 4, H.mass_off.size() * 8,
-                            H.br_nblk.size() * 4,              0};
+                            H.br_nblk.size() * 4,              0,
+                            H.seg_block_off.size() * 4,        H.seg_sharer_off.size() * 4,
+                            H.score_chunks.size() * 4};
     size_t offs[kN], off = 0;
     for (int i = 0; i < kN; ++i) {
         offs[i] = off;
@@ -199,6 +203,9 @@ int32_t upload_plan(rksc_plan* p) {
     p->dev.mass_off = reinterpret_cast<const int64_t*>(base + offs[5]);
     p->dev.br_nblk = reinterpret_cast<const int32_t*>(base + offs[6]);
     p->dev.counters = reinterpret_cast<int32_t*>(base + offs[7]);
+    p->dev.seg_block_off = reinterpret_cast<const int32_t*>(base + offs[8]);
+    p->dev.seg_sharer_off = reinterpret_cast<const int32_t*>(base + offs[9]);
+    p->dev.score_chunks = reinterpret_cast<const int32_t*>(base + offs[10]);
     p->on_device = true;
     return RKSC_OK;
 }
@@ -575,4 +582,55 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_static(const rksc_plan*
     if (st != RKSC_OK) return st;
     return rksc_branch_decode_attention(plan, q, k_pool, v_pool, out, block_mass, ws,
                                         (size_t)RKSC_STATIC_WORKSPACE_BYTES, device_status, stream);
+}
+
+// ---- RSBCM eviction (Section 2.4, Algorithm 4) ----
+
+extern "C" RKSC_API int32_t rksc_rsbcm_page_scores(const rksc_plan* plan, const float* block_mass, double* score,
+                                                   void* stream) {
+    if (!plan) return RKSC_ERR_INVALID_ARG;
+    const HostPlan& H = plan->host;
+    const int num_chunks = (int)(H.score_chunks.size() / 2);
+    if (num_chunks == 0) return RKSC_OK;
+    if (!block_mass || !score || !plan->on_device) return RKSC_ERR_INVALID_ARG;
+    int32_t st = ensure_device(nullptr);
+    if (st != RKSC_OK) return st;
+    cudaError_t e = launch_page_scores(reinterpret_cast<const int2*>(plan->dev.score_chunks), num_chunks,
+                                       plan->dev.seg_block_off, plan->dev.seg_sharer_off, plan->dev.sharers, block_mass,
+                                       score, H.layout.num_q_heads, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda = e;
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    return RKSC_OK;
+}
+
+extern "C" RKSC_API size_t rksc_rsbcm_workspace_bytes(int64_t n) {
+    if (n < 0) n = 0;
+    const size_t b = ((size_t)n * 8 + 255) / 256 * 256;
+    return b ? b : 256;
+}
+
+extern "C" RKSC_API int32_t rksc_rsbcm_evict(const double* score, const int32_t* depth, int64_t n, int64_t capacity,
+                                             uint8_t* evicted, int32_t* num_evicted, void* workspace,
+                                             size_t workspace_bytes, void* stream) {
+    if (n < 0 || n >= ((int64_t)1 << 31)) return RKSC_ERR_INVALID_ARG;
+    if (n > 0 && (!score || !depth || !evicted)) return RKSC_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < rksc_rsbcm_workspace_bytes(n) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
+        return RKSC_ERR_WORKSPACE;
+    if (n == 0 && !num_evicted) return RKSC_OK;
+    int32_t st = ensure_device(nullptr);
+    if (st != RKSC_OK) return st;
+    if (capacity < 0) capacity = 0;
+    const uint32_t k = capacity >= n ? 0u : (uint32_t)(n - capacity);
+    cudaError_t e = launch_rsbcm_select(score, depth, (int32_t)n, k, static_cast<uint64_t*>(workspace), evicted,
+                                        num_evicted, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda = e;
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    return RKSC_OK;
 }

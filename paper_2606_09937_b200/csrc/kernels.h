@@ -42,4 +42,12 @@ cudaError_t launch_seg_attn_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                cudaStream_t stream);
 cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream);
 
+// RSBCM (Section 2.4, Algorithm 4): per-entry scores from the block masses; exact selection of the
+// k entries smallest by (score / (depth + 1), index).  keys: scratch of n 64-bit words.
+cudaError_t launch_page_scores(const int2* chunks, int num_chunks, const int32_t* seg_block_off,
+                               const int32_t* seg_sharer_off, const Sharer* sharers, const float* mass, double* score,
+                               int Hq, cudaStream_t stream);
+cudaError_t launch_rsbcm_select(const double* score, const int32_t* depth, int32_t n, uint32_t k, uint64_t* keys,
+                                uint8_t* evicted, int32_t* num_evicted, cudaStream_t stream);
+
 }  // namespace rksc

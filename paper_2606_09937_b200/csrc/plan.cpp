@@ -244,6 +244,15 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
             }
     }
 
+    // grid of the page-score kernel (RSBCM): 32 consecutive pages of one segment per CTA
+    for (int s = 0; s < S; ++s) {
+        const int n = P.seg_block_off[s + 1] - P.seg_block_off[s];
+        for (int p0 = 0; p0 < n; p0 += 32) {
+            P.score_chunks.push_back(s);
+            P.score_chunks.push_back(p0);
+        }
+    }
+
     // workspace: partial outputs [rows][d] fp32, then partial log2-sum-exp [rows] fp32
     const size_t o_bytes = ((size_t)P.num_partial_rows * L.head_dim * sizeof(float) + 255) / 256 * 256;
     P.ws_lse_offset = o_bytes;
@@ -330,4 +339,60 @@ extern "C" RKSC_API void rksc_tables_free(rksc_tables* t) {
     std::free((void*)t->br_seg_off);
     std::free((void*)t->br_segs);
     std::memset(t, 0, sizeof(*t));
+}
+
+// Tables after RSBCM eviction (Algorithm 4's effect on the block tables).
+extern "C" RKSC_API int32_t rksc_tables_drop_evicted(const rksc_tables* in, const uint8_t* evicted, rksc_tables* out) {
+    if (!in || !out) return RKSC_ERR_INVALID_ARG;
+    std::memset(out, 0, sizeof(*out));
+    const int B = in->num_branches, S = in->num_segments;
+    if (B < 0 || S < 0 || !in->seg_block_off || !in->br_seg_off) return RKSC_ERR_INVALID_ARG;
+    if (S > 0 && !in->seg_num_tokens) return RKSC_ERR_INVALID_ARG;
+    if (in->seg_block_off[0] != 0 || in->br_seg_off[0] != 0) return RKSC_ERR_BAD_TABLE;
+    for (int s = 0; s < S; ++s) {
+        const int64_t n = (int64_t)in->seg_block_off[s + 1] - in->seg_block_off[s];
+        const int64_t nt = in->seg_num_tokens[s];
+        if (n < 0 || nt < 0 || nt > n * rksc::kBlock || nt <= (n - 1) * rksc::kBlock) {
+            if (!(n == 0 && nt == 0)) return RKSC_ERR_BAD_TABLE;
+        }
+    }
+    for (int b = 0; b < B; ++b)
+        if (in->br_seg_off[b + 1] < in->br_seg_off[b]) return RKSC_ERR_BAD_TABLE;
+    const int64_t N = in->seg_block_off[S], R = in->br_seg_off[B];
+    if (N > 0 && (!in->seg_blocks || !evicted)) return RKSC_ERR_INVALID_ARG;
+    if (R > 0 && !in->br_segs) return RKSC_ERR_INVALID_ARG;
+    auto alloc = [](size_t n) { return (int32_t*)std::malloc(std::max<size_t>(1, n) * sizeof(int32_t)); };
+    int32_t* a0 = alloc((size_t)S + 1);
+    int32_t* a1 = alloc((size_t)N);
+    int32_t* a2 = alloc((size_t)S);
+    int32_t* a3 = alloc((size_t)B + 1);
+    int32_t* a4 = alloc((size_t)R);
+    if (!a0 || !a1 || !a2 || !a3 || !a4) {
+        std::free(a0); std::free(a1); std::free(a2); std::free(a3); std::free(a4);
+        return RKSC_ERR_NOMEM;
+    }
+    int32_t kept = 0;
+    a0[0] = 0;
+    for (int s = 0; s < S; ++s) {
+        const int lo = in->seg_block_off[s], hi = in->seg_block_off[s + 1];
+        const int ntok = in->seg_num_tokens[s];
+        int kept_tok = 0;
+        for (int p = 0; p < hi - lo; ++p) {
+            if (evicted[lo + p]) continue;
+            a1[kept++] = in->seg_blocks[lo + p];
+            kept_tok += std::min(rksc::kBlock, ntok - p * rksc::kBlock);
+        }
+        a0[s + 1] = kept;
+        a2[s] = kept_tok;
+    }
+    std::memcpy(a3, in->br_seg_off, ((size_t)B + 1) * sizeof(int32_t));
+    if (R > 0) std::memcpy(a4, in->br_segs, (size_t)R * sizeof(int32_t));
+    out->num_branches = B;
+    out->num_segments = S;
+    out->seg_block_off = a0;
+    out->seg_blocks = a1;
+    out->seg_num_tokens = a2;
+    out->br_seg_off = a3;
+    out->br_segs = a4;
+    return RKSC_OK;
 }

@@ -51,6 +51,9 @@ struct DevicePlan {
     const int32_t* merge_rows = nullptr;  // partial row of head-in-group 0 for each part
     const int64_t* mass_off = nullptr;    // [B+1]
     const int32_t* br_nblk = nullptr;     // [B]
+    const int32_t* seg_block_off = nullptr;   // [S+1]
+    const int32_t* seg_sharer_off = nullptr;  // [S+1]
+    const int32_t* score_chunks = nullptr;    // (segment, first page) pairs, 32 pages each: the score kernel's grid
     int32_t* counters = nullptr;          // [4] work-claim counters (warp kernel, tcgen05 kernel), zero between launches
 };
 
@@ -67,6 +70,7 @@ struct HostPlan {
     std::vector<int32_t> seg_sharer_off;  // [S+1]
     std::vector<int32_t> merge_off;
     std::vector<int32_t> merge_rows;
+    std::vector<int32_t> score_chunks;    // (segment, first page) pairs of the page-score kernel
     std::vector<int64_t> mass_off;        // [B+1]
     std::vector<int32_t> br_nblk;         // [B]
     int64_t mass_elems = 0;
@@ -92,6 +96,7 @@ struct HostPlan {
         seg_sharer_off.clear();
         merge_off.clear();
         merge_rows.clear();
+        score_chunks.clear();
         mass_off.clear();
         br_nblk.clear();
         mass_elems = 0;

@@ -24,6 +24,8 @@ from .generators import (  # noqa: F401
     make_long_context,
     punch_holes,
     lowest_mass_pages,
+    make_block_masses,
+    make_eviction_inputs,
     unique_kv_bytes,
     duplicated_kv_bytes,
     CONFIG_NAMES,

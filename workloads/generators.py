@@ -417,6 +417,33 @@ def punch_holes(w: Workload, segment: int, evicted_logical_pages: np.ndarray) ->
     return out
 
 
+def make_block_masses(t: Tables, num_q_heads: int, seed: int = SEED_BASE + 50) -> list:
+    """Synthetic stand-ins for the attention's second output: for every branch an fp32 array
+    [Hq][nblk_b] of non-negative numbers, each row scaled to sum to about 1, with the heavy
+    tail real softmax masses have (a few blocks take most of the mass, many are near zero)."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for b in range(t.num_branches):
+        segs = t.br_segs[t.br_seg_off[b]:t.br_seg_off[b + 1]]
+        nblk = int(sum(int(t.seg_block_off[s + 1] - t.seg_block_off[s]) for s in segs))
+        m = np.exp(4.0 * rng.standard_normal((num_q_heads, nblk)))
+        m /= np.maximum(m.sum(axis=1, keepdims=True), 1e-300)
+        out.append(m.astype(np.float32))
+    return out
+
+
+def make_eviction_inputs(n: int, seed: int = SEED_BASE + 51, max_depth: int = 6, tie_levels: int = 0):
+    """(score fp64 [n] >= 0, depth int32 [n]) for an eviction.  tie_levels > 0 draws the scores from
+    that many distinct values, so that many entries share one omega."""
+    rng = np.random.default_rng(seed)
+    if tie_levels > 0:
+        score = rng.integers(0, tie_levels, n).astype(np.float64) / 8.0
+    else:
+        score = np.exp(3.0 * rng.standard_normal(n))
+    depth = rng.integers(0, max_depth + 1, n).astype(np.int32)
+    return score, depth
+
+
 def make_config(name: str, **kw) -> Workload:
     if name == "tiny":
         return make_tiny(**kw)
