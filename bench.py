@@ -503,6 +503,11 @@ def run_ours(args):
             "pct_of_measured_copy_peak": 100.0 * kv_bytes / (med * 1e-3) / 1e9 / peak_gbs,
             "branch_steps_per_s": B / (med * 1e-3),
         }
+        # RSBCM (Section 2.4, Algorithm 4) on this step's masses: every listed page competes, N_max = 2000
+        _, info = rsbcm_pass(rk, batch, plan, batch.mass, slice(0, plan.num_pages_listed), 2000)
+        info["what"] = ("after a step, outside the timed region: rksc_rsbcm_page_scores over the step's block masses, "
+                        "then rksc_rsbcm_evict down to the paper's default capacity of 2000 entries")
+        line["rsbcm"] = info
         if not args.no_e2e and batch.has_gate:
             line["e2e"] = run_e2e(rk, batch, kv_bytes, args.e2e_steps)
         if not args.no_sweep:
@@ -578,8 +583,47 @@ def aggregate_over_ranks(dist, dev, kv_bytes: int, steps: int, total_ms: float):
     return float(b.item()) * steps / (total_ms_max * 1e-3) / 1e12, total_ms_max
 
 
+def _event_us(fn, iters=20):
+    import torch
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / iters
+
+
+def rsbcm_pass(rk, batch: DeviceBatch, plan, mass, entries: slice, capacity: int, timed: bool = True):
+    """RSBCM on the masses of a finished step (Section 2.4, Algorithm 4), all on the GPU: page scores,
+    then the eviction among `entries` (depth 0) down to `capacity`.  Returns (host mask over all the
+    plan's entries, timing dict)."""
+    import torch
+    n_all = plan.num_pages_listed
+    score = rk.rksc_rsbcm_page_scores(plan, mass)
+    sub = score[entries]
+    n = int(sub.numel())
+    depth = torch.zeros(n, dtype=torch.int32, device=score.device)
+    ev = torch.empty(n, dtype=torch.uint8, device=score.device)
+    cnt = torch.empty(1, dtype=torch.int32, device=score.device)
+    ws = torch.empty(rk.rksc_rsbcm_workspace_bytes(n), dtype=torch.uint8, device=score.device)
+    rk.rksc_rsbcm_evict(sub, depth, capacity, ev, cnt, ws)
+    torch.cuda.synchronize()
+    mask = np.zeros(n_all, dtype=np.uint8)
+    mask[entries] = ev.cpu().numpy()
+    info = {"entries": n, "capacity": int(capacity), "evicted": int(cnt.item())}
+    if timed:
+        info["page_scores_us"] = _event_us(lambda: rk.rksc_rsbcm_page_scores(plan, mass, score))
+        info["evict_us"] = _event_us(lambda: rk.rksc_rsbcm_evict(sub, depth, capacity, ev, cnt, ws))
+    return mask, info
+
+
 def punch_long_context(rk, batch: DeviceBatch):
-    """Config 5: evict the 20 % of prefix pages with the lowest mass of a prior full-table step (computed on the GPU)."""
+    """Config 5: the 20 % of the prefix pages with the lowest attention mass of a prior full-table step are
+    evicted - scores, selection and holed tables all by the library's RSBCM calls."""
     import torch
     import workloads
     w = batch.w
@@ -589,12 +633,15 @@ def punch_long_context(rk, batch: DeviceBatch):
                                                  block_mass=batch.mass, workspace=batch.workspace,
                                                  device_status=batch.status)
     torch.cuda.synchronize()
-    masses = rk.split_block_mass(plan, mass)
     npg = int(w.tables.seg_block_off[1])
-    scores = sum(m[:, :npg].astype(np.float64).sum(axis=0) for m in masses)
-    holed = workloads.punch_holes(w, 0, workloads.lowest_mass_pages(scores, 0.2))
-    batch.w = holed
-    batch.tables = rk.Tables.of(holed.tables)
+    mask, info = rsbcm_pass(rk, batch, plan, mass, slice(0, npg), npg - int(0.2 * npg))
+    holed = rk.rksc_tables_drop_evicted(w.tables, mask)
+    t = workloads.Tables(seg_block_off=holed.seg_block_off, seg_blocks=holed.seg_blocks,
+                         seg_num_tokens=holed.seg_num_tokens, br_seg_off=holed.br_seg_off, br_segs=holed.br_segs)
+    import dataclasses
+    batch.w = dataclasses.replace(w, tables=t, flat=None)
+    batch.tables = holed
+    return info
 
 
 def sweep_configs(rk, dev, flush, peak_gbs, skip, cached):
@@ -609,8 +656,7 @@ def sweep_configs(rk, dev, flush, peak_gbs, skip, cached):
             continue
         w = load_workload(name)
         b = DeviceBatch(w, dev)
-        if name == "long_context":
-            punch_long_context(rk, b)
+        rsbcm = punch_long_context(rk, b) if name == "long_context" else None
         plan, _ = run_step(rk, b)
         torch.cuda.synchronize()
         kv, _ = algorithmic_bytes(plan, b.w.layout)
@@ -620,6 +666,8 @@ def sweep_configs(rk, dev, flush, peak_gbs, skip, cached):
                      "tbps_unique_kv": kv / (med * 1e-3) / 1e12,
                      "pct_of_8tbps": 100.0 * kv / (med * 1e-3) / 1e12 / NOMINAL_HBM_TBPS,
                      "branch_steps_per_s": b.w.num_branches / (med * 1e-3), "work_items": plan.num_work_items}
+        if rsbcm is not None:
+            res[name]["rsbcm_eviction_before_this_step"] = rsbcm
         del b
         torch.cuda.empty_cache()
     return res
