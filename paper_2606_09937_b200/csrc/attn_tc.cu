@@ -5,24 +5,28 @@
 // 128 rows of one MMA tile; a KV page staged in shared memory once then serves every sharing
 // branch (the shared-prefix read that replaces the paper's per-branch copies of the prefix cache,
 // Algorithm 1 line 3 / Section 2.2).  Here the product really is a dense contraction:
-//   S[128 x 64]  = Q[128 x d] K^T        (tcgen05.mma, A = Q read from tensor memory, B = K slot, K-major,
-//                                         in 128-byte-swizzled smem)
+//   S[128 x 64]  = Q[128 x d] K^T        (tcgen05.mma, A = Q and B = K slot, both K-major in
+//                                         128-byte-swizzled shared memory)
 //   O[128 x d]  += P[128 x 64] V         (A = P read from tensor memory, B = V MN-major in smem)
-// with Q, S, P and O in tensor memory.  One persistent CTA per SM, eleven warps:
+// with S, P and O in tensor memory.  One persistent CTA per SM, twelve warps:
 //   warps 0-3 / 4-7  two softmax warpgroups; thread = one stacked row (TMEM lane).  They take
-//                    alternate 64-token slots of an item, each with its own S and O accumulator and
+//                    alternate 64-token slots, each with two S buffers, its own O accumulator and
 //                    its own running (max, sum), merged at the end of the item.  Per slot: tcgen05.ld
 //                    of the S row, scale + mask + online softmax in base 2, per-page softmax mass
-//                    (log2, absolute) to global memory, P as bf16 back to tensor memory (tcgen05.st);
-//                    O is rescaled in TMEM (tcgen05.ld / st) only when a running maximum of the warp moved.
-//   warp 8           producer: claims work items from a global counter and streams their pages by
-//                    TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a five-slot
-//                    ring, four pages per slot, with a header per slot that the other warps follow.
-//   warps 9, 10      MMA issuers, one per warpgroup (one lane each; warp 9 also allocates TMEM): S of the
-//                    warpgroup's next slot is issued before P V of its previous one, so S is waiting when
-//                    the warpgroup comes out of its softmax and the tensor pipe runs under both softmaxes.
-// Completion of MMAs is signalled with tcgen05.commit onto mbarriers (S ready, O ready / P free,
-// ring slot free).  Every wait is bounded: on expiry the CTA records RKSC_ERR_DEVICE_TIMEOUT,
+//                    (log2, absolute) to global memory, P as bf16 written over the first half of the
+//                    same S buffer (tcgen05.st); O is rescaled in TMEM only when a running maximum
+//                    of the warp moved by more than 2^8.  A warpgroup's only wait per slot is "S ready".
+//   warp 8           producer: claims work items from a global counter, publishes their descriptors
+//                    in a small item ring and streams their pages by TMA (cp.async.bulk.tensor,
+//                    128-byte swizzle, no multicast) into a five-slot ring, four pages per slot.
+//   warps 9, 10      MMA issuers, one per warpgroup (one lane each; warp 9 also allocates TMEM): S of
+//                    the warpgroup's next slot is issued before P V of its previous one, into the S
+//                    buffer that P V before that has read, so S is waiting when the warpgroup comes
+//                    out of its softmax and the tensor pipe runs under both softmaxes.
+//   warp 11          Q loader: an item ahead, gathers the item's stacked query rows into the
+//                    swizzled Q tile (cp.async) and each row's block-mass base into shared memory.
+// Completion of MMAs is signalled with tcgen05.commit onto mbarriers (S ready, P V done / ring slot
+// free, Q tile free).  Every wait is bounded: on expiry the CTA records RKSC_ERR_DEVICE_TIMEOUT,
 // stops issuing work, skips further waits, frees its TMEM and returns.
 #include <cuda_bf16.h>
 
@@ -36,46 +40,58 @@ constexpr int HD = 128;
 constexpr int kSmWarps = 8;                       // softmax warps (two warpgroups)
 constexpr int kProducerWarp = kSmWarps;           // 8
 constexpr int kMmaWarp = kSmWarps + 1;            // 9 and 10: MMA issuers of warpgroup 0 and 1
-constexpr int kTcThreads = (kSmWarps + 3) * 32;   // 352
-constexpr int kNS = 6;                            // ring slots
+constexpr int kQWarp = kSmWarps + 3;              // 11: Q loader
+constexpr int kVWarp = kSmWarps + 4;              // 12, 13, 14: follower producers (V even slots, K odd, V odd)
+constexpr int kTcThreads = (kSmWarps + 8) * 32;   // 512: four warpgroups (warp 15 idles), so that registers can be re-divided
+constexpr int kNK = 4;                            // K ring slots (even: a slot always serves the same warpgroup)
+constexpr int kNV = 4;                            // V ring slots (even)
+constexpr int kVLag = 4;                          // the V stream runs this many slots behind the K stream
+constexpr int kNI = 4;                            // item ring entries
 constexpr int kSlotTokens = 64;                   // 4 pages
 constexpr int kKBytes = kSlotTokens * HD * 2;     // K (or V) of a slot: [half][64 tokens][128 B] = 16 KiB
-constexpr int kSlotBytes = 2 * kKBytes;
-constexpr int kRingBytes = kNS * kSlotBytes;      // 192 KiB
-constexpr int kMlOff = kRingBytes;                // (m, l) exchange [2][128] float2
-constexpr int kBarOff = kMlOff + 2 * 128 * 8;
+constexpr int kVOff = kNK * kKBytes;
+constexpr int kRingBytes = (kNK + kNV) * kKBytes; // 128 KiB
+static_assert(kNK % 2 == 0 && kNV % 2 == 0 && kVLag >= 1 && kVLag < kNK + 4 && kVLag < 8, "ring geometry");
+constexpr int kQOff = kRingBytes;                 // Q tiles [2 (item parity)][half][128 rows][128 B], 128-byte swizzle: 2 x 32 KiB
+constexpr int kQBytes = 128 * HD * 2;
+constexpr int kRowOff = kQOff + 2 * kQBytes;      // block-mass base of every row [2][128] int64
+constexpr int kMlOff = kRowOff + 2 * 128 * 8;     // (m, l) exchange [2 (item parity)][2 (warpgroup)][128] float2
+constexpr int kBarOff = kMlOff + 2 * 2 * 128 * 8;
 // mbarriers
-constexpr int kBarFull = 0;                       // [kNS]  producer -> everyone: slot landed (+ header)
-constexpr int kBarEmpty = kBarFull + kNS;         // [kNS]  slot reusable: P V committed + 10 header readers
-constexpr int kBarSFull = kBarEmpty + kNS;        // [2]    S of the warpgroup's slot is in TMEM
-constexpr int kBarSFree = kBarSFull + 2;          // [2]    the warpgroup has copied S to registers
-constexpr int kBarPFull = kBarSFree + 2;          // [2]    P of the slot is in tensor memory
-constexpr int kBarODone = kBarPFull + 2;          // [2]    P V of the slot has completed
-constexpr int kBarQFull = kBarODone + 2;          // Q tile of the item is in tensor memory
-constexpr int kBarEpiA = kBarQFull + 1;           // item epilogue: (m, l) published
-constexpr int kBarEpiB = kBarEpiA + 1;            // item epilogue: accumulators read
+constexpr int kBarFullK = 0;                      // [kNK]  producer -> issuer: K of the slot landed
+constexpr int kBarEmptyK = kBarFullK + kNK;       // [kNK]  K slot reusable: its Q K^T has completed
+constexpr int kBarFullV = kBarEmptyK + kNK;       // [kNV]  V of the slot landed
+constexpr int kBarEmptyV = kBarFullV + kNV;       // [kNV]  V slot reusable: its P V has completed
+constexpr int kBarItemFull = kBarEmptyV + kNV;    // [kNI]  item descriptor published
+constexpr int kBarItemEmpty = kBarItemFull + kNI; // [kNI]  ... read by the 8 softmax warps, 2 issuers, Q loader
+constexpr int kBarQFull = kBarItemEmpty + kNI;    // [2]    Q tile and row bases of the item are in shared memory
+constexpr int kBarQEmpty = kBarQFull + 2;         // [2]    every Q K^T of the item has completed (both issuers) and
+                                                  //        the softmax warps have read their row bases
+constexpr int kBarSFull = kBarQEmpty + 2;         // [2][2] S of the warpgroup's slot is in its buffer
+constexpr int kBarPFull = kBarSFull + 4;          // [2][2] P of the slot is in the buffer
+constexpr int kBarODone = kBarPFull + 4;          // [2]    P V of the warpgroup's slot has completed
+constexpr int kBarEpiA = kBarODone + 2;           //        item epilogue: (m, l) published
+constexpr int kBarEpiB = kBarEpiA + 1;            //        item epilogue: accumulators read
 constexpr int kNumBars = kBarEpiB + 1;
-constexpr int kHdrOff = kBarOff + ((kNumBars * 8 + 15) / 16) * 16;
-constexpr int kTmemPtrOff = kHdrOff + kNS * 64;
+constexpr int kItemOff = kBarOff + ((kNumBars * 8 + 15) / 16) * 16;
+constexpr int kVInfoOff = kItemOff + kNI * 64;    // [8] slots the K stream has issued and the V stream has not: 4 page ids, pages, KV head
+constexpr int kTmemPtrOff = kVInfoOff + 8 * 32;
 constexpr int kFlagOff = kTmemPtrOff + 16;
 constexpr int kSmemTotal = kFlagOff + 16;
+static_assert(kSmemTotal + 1024 <= 227 * 1024, "shared memory of the tcgen05 kernel");
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;                     // S[wg]: 64 fp32 columns at 64*wg
-constexpr uint32_t kColO = 128;                   // O[wg]: 128 fp32 columns at 128 + 128*wg
-constexpr uint32_t kColP = 384;                   // P[wg]: 64 bf16 = 32 columns at 384 + 32*wg
-constexpr uint32_t kColQ = 448;                   // Q: 128 bf16 per row = 64 columns (half wg written by warpgroup wg)
+constexpr uint32_t kColS = 0;                     // S[wg][buf]: 64 fp32 columns at 64 * (2 * wg + buf); P over its first 32
+constexpr uint32_t kColO = 256;                   // O[wg]: 128 fp32 columns at 256 + 128 * wg
 constexpr float kRescaleStep = 8.f;               // O is rescaled only when a row's max moved by more than 2^8
 
-struct __align__(16) SlotHeader {
+struct __align__(16) ItemHeader {
     int32_t item;        // index of the work item, -1: no more work
-    int32_t group;       // position of this slot within the item (0 = first)
-    int32_t num_pages;   // pages staged in this slot (1..4)
-    int32_t last;        // 1 on the item's last slot
+    int32_t num_groups;  // 64-token slots of the item
+    int32_t pad0, pad1;
     WorkItem it;
-    int32_t num_groups;  // slots of the item
-    int32_t pad;
+    int32_t pad2, pad3;
 };
-static_assert(sizeof(SlotHeader) == 64, "SlotHeader is 64 bytes");
+static_assert(sizeof(ItemHeader) == 64, "ItemHeader is 64 bytes");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -174,6 +190,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -188,20 +213,46 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// A and B operands from shared memory
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+#ifdef EXP_STREAMONLY
+#define umma_ss(...)
+#define umma_ts(...)
+#define tc_commit(b) mbar_arrive(b)
+#endif
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
 #ifdef RKSC_WAIT_PROFILE
-// Development aid: cycles per CTA spent in the waits of the MMA lane ([0..4]: total, slot landed,
-// S buffer free, P ready, Q ready) and of softmax warp 0 ([8..15]: total, slot landed, S ready,
-// previous P V done, epilogue A, epilogue B, slots, items).
-__device__ unsigned long long g_tc_prof[384][16];
-#define TCPROF_DECL unsigned long long tcp[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long tcp_begin = clock64()
-#define TCPROF_WAIT(i, stmt) { const long long _t = clock64(); stmt; tcp[i] += (unsigned long long)(clock64() - _t); }
-#define TCPROF_MARK(i) { const long long _n = clock64(); tcq[i] += (unsigned long long)(_n - tcq_t); tcq_t = _n; }
-#define TCPROF_FLUSH(base) { tcp[0] = (unsigned long long)(clock64() - tcp_begin); for (int _i = 0; _i < 8; ++_i) g_tc_prof[blockIdx.x][base + _i] = tcp[_i]; }
+// Development aid: cycles one lane of each role spent in its waits.
+__device__ unsigned long long g_tc_prof[160][32];
+__device__ long long g_tc_trace[4][2048];
+__device__ int g_tc_trace_n[4];
+#define TCTRACE_DECL(w_) int tr_n = 0; const bool tr_on = blockIdx.x == 0 && (threadIdx.x & 31) == 0; long long* const tr_buf = g_tc_trace[w_]
+#define TCTRACE(ev) { if (tr_on && tr_n < 2048) { tr_buf[tr_n++] = (clock64() << 12) | (long long)((ev) & 4095); } }
+#define TCTRACE_END(w_) { if (tr_on) g_tc_trace_n[w_] = tr_n; }
+__device__ int g_tc_dbg[32][4];
+__device__ int g_tc_dbg_n, g_tc_dbg_n2;
+#define TCP_DECL unsigned long long tcp[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long tcp_begin = clock64()
+#define TCP_WAIT(i, stmt) { const long long _t = clock64(); stmt; tcp[i] += (unsigned long long)(clock64() - _t); }
+#define TCP_FLUSH(base) { tcp[0] = (unsigned long long)(clock64() - tcp_begin); for (int _i = 0; _i < 8; ++_i) g_tc_prof[blockIdx.x][base + _i] = tcp[_i]; }
 #else
-#define TCPROF_DECL
-#define TCPROF_WAIT(i, stmt) stmt
-#define TCPROF_MARK(i)
-#define TCPROF_FLUSH(base)
+#define TCP_DECL
+#define TCP_WAIT(i, stmt) stmt
+#define TCP_FLUSH(base)
+#define TCTRACE_DECL(w_)
+#define TCTRACE(ev)
+#define TCTRACE_END(w_)
 #endif
 
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -212,23 +263,35 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bars = sbase + kBarOff;
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
-    SlotHeader* s_hdr = reinterpret_cast<SlotHeader*>(smem + kHdrOff);
+    ItemHeader* s_item = reinterpret_cast<ItemHeader*>(smem + kItemOff);
+    int64_t* s_rowbase = reinterpret_cast<int64_t*>(smem + kRowOff);
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + kTmemPtrOff);
     volatile int32_t* s_abort = reinterpret_cast<volatile int32_t*>(smem + kFlagOff);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int i = 0; i < kNS; ++i) {
-            mbar_init(bar(kBarFull + i), 1);
-            mbar_init(bar(kBarEmpty + i), 1 + kSmWarps + 2);   // P V commit, 8 softmax warps, 2 MMA issuers
+        for (int i = 0; i < kNK; ++i) {
+            mbar_init(bar(kBarFullK + i), 1);
+            mbar_init(bar(kBarEmptyK + i), 1);
         }
-        for (int w = 0; w < 2; ++w) {
-            mbar_init(bar(kBarSFull + w), 1);
-            mbar_init(bar(kBarSFree + w), 4);
-            mbar_init(bar(kBarPFull + w), 4);
-            mbar_init(bar(kBarODone + w), 1);
+        for (int i = 0; i < kNV; ++i) {
+            mbar_init(bar(kBarFullV + i), 1);
+            mbar_init(bar(kBarEmptyV + i), 1);
         }
-        mbar_init(bar(kBarQFull), kSmWarps);
+        for (int i = 0; i < kNI; ++i) {
+            mbar_init(bar(kBarItemFull + i), 1);
+            mbar_init(bar(kBarItemEmpty + i), kSmWarps + 6);   // 8 softmax warps, 2 issuers, Q loader, 3 follower producers
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(kBarQFull + i), 1);
+            mbar_init(bar(kBarQEmpty + i), 2 + kSmWarps);
+        }
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(bar(kBarSFull + i), 1);
+            mbar_init(bar(kBarPFull + i), 4);
+        }
+        mbar_init(bar(kBarODone + 0), 1);
+        mbar_init(bar(kBarODone + 1), 1);
         mbar_init(bar(kBarEpiA), kSmWarps);
         mbar_init(bar(kBarEpiB), kSmWarps);
         *s_abort = 0;
@@ -250,11 +313,21 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     auto wait_or_abort = [&](uint32_t b, uint32_t parity) {
         if (*s_abort) return;
         if (!mbar_wait(b, parity)) {
+#ifdef RKSC_WAIT_PROFILE
+            if (!*s_abort && atomicAdd(&g_tc_dbg_n, 1) < 32) {
+                const int k_ = atomicAdd(&g_tc_dbg_n2, 1);
+                if (k_ < 32) { g_tc_dbg[k_][0] = (b - bars) / 8; g_tc_dbg[k_][1] = parity; g_tc_dbg[k_][2] = warp; g_tc_dbg[k_][3] = blockIdx.x; }
+            }
+#endif
             *s_abort = 1;
             if (a.status) atomicExch(a.status, RKSC_ERR_DEVICE_TIMEOUT);
         }
     };
 
+    // 512 threads leave 128 registers each; the two softmax warpgroups need more and the two
+    // warpgroups of helper warps much less
+    if (warp >= kSmWarps) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
     if (warp == kProducerWarp) {
         // ------------------------------------ producer ------------------------------------
         auto claim = [&]() {
@@ -270,62 +343,67 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         auto fetch_ids = [&](const WorkItem& w, int first) {
             return (first + lane < w.num_pages) ? __ldg(a.plan.seg_blocks + w.page_begin + first + lane) : 0;
         };
-        // One item is claimed ahead of the one being streamed (its descriptor and first page ids are
-        // fetched while this one streams); claiming further ahead would starve other CTAs, there
-        // being only a few of these long items per CTA.
+        TCP_DECL;
+        TCTRACE_DECL(2);
+        int nitem = 0;   // item descriptors published
+        auto publish = [&](int idx, const WorkItem& w) {
+            const int e = nitem % kNI;
+            if (nitem >= kNI) wait_or_abort(bar(kBarItemEmpty + e), (uint32_t)(nitem / kNI - 1) & 1u);
+            if (lane == 0) {
+                ItemHeader h{};
+                h.item = idx < a.num_tc_items ? idx : -1;
+                h.num_groups = (w.num_pages + 3) / 4;
+                h.it = w;
+                s_item[e] = h;
+                mbar_arrive(bar(kBarItemFull + e));
+            }
+            __syncwarp();
+            ++nitem;
+        };
+        // One item is claimed ahead of the one being streamed (its descriptor is published, so the Q
+        // loader can fetch its rows, and its first page ids are fetched while this one streams);
+        // claiming further ahead would starve other CTAs, there being only a few of these long
+        // items per CTA.
+        // K and V travel in rings of their own, each fed by its own warp (one warp cannot issue TMA
+        // copies fast enough for the whole stream): K of a slot is needed two slots before its softmax
+        // starts and is free again as soon as Q K^T has run, V is needed after the softmax.
         int seq = 0;
         int idx = claim();
         WorkItem it = fetch_item(idx);
+        publish(idx, it);
         int ids = fetch_ids(it, 0);
         while (idx < a.num_tc_items && !*s_abort) {
             const int nidx = claim();
             const WorkItem nit = fetch_item(nidx);
+            publish(nidx, nit);     // past the last item this is the end marker
             const int ngroups = (it.num_pages + 3) / 4;
             int ids_ahead = 0;
             for (int g = 0; g < ngroups; ++g, ++seq) {
-                const int slot = seq % kNS;
+                const int kslot = seq % kNK;
                 const int npg = min(4, it.num_pages - g * 4);
                 if ((g & 7) == 0) ids_ahead = fetch_ids(it, (g + 8) * 4);
-                const int page = __shfl_sync(0xffffffffu, ids, (g & 7) * 4 + (lane & 3));
+                // lane = 2 * page + half
+                const int page = __shfl_sync(0xffffffffu, ids, (g & 7) * 4 + ((lane >> 1) & 3));
                 if ((g & 7) == 7) ids = ids_ahead;
-                if (seq >= kNS) wait_or_abort(bar(kBarEmpty + slot), (uint32_t)(seq / kNS - 1) & 1u);
+                if (seq & 1) continue;   // odd slots: warp 13
+                TCTRACE(1024 + (seq & 1023));
+                if (seq >= kNK) TCP_WAIT(1, wait_or_abort(bar(kBarEmptyK + kslot), (uint32_t)(seq / kNK - 1) & 1u));
                 if (*s_abort) break;
-                const uint32_t full = bar(kBarFull + slot);
-                if (lane == 0) {
-                    SlotHeader h;
-                    h.item = idx;
-                    h.group = g;
-                    h.num_pages = npg;
-                    h.last = (g == ngroups - 1);
-                    h.it = it;
-                    h.num_groups = ngroups;
-                    h.pad = 0;
-                    s_hdr[slot] = h;
-                    mbar_arrive_expect_tx(full, npg * 2 * (kBlock * HD * 2));
-                }
+                TCTRACE(seq & 1023);
+                const uint32_t full = bar(kBarFullK + kslot);
+                if (lane == 0) mbar_arrive_expect_tx(full, npg * (kBlock * HD * 2));
                 __syncwarp();
-                if (lane < npg) {
+                if (lane < npg * 2) {
                     const int y = (page * a.Hkv + it.kv_head) * kBlock;
-                    const uint32_t kdst = sbase + slot * kSlotBytes + lane * 2048;
-#pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
-                        tma_load_2d(kdst + hh * 8192, &tm_k, hh * 64, y, full);
-                        tma_load_2d(kdst + kKBytes + hh * 8192, &tm_v, hh * 64, y, full);
-                    }
+                    tma_load_2d(sbase + kslot * kKBytes + (lane >> 1) * 2048 + (lane & 1) * 8192, &tm_k, (lane & 1) * 64, y, full);
                 }
             }
             idx = nidx;
             it = nit;
             ids = fetch_ids(it, 0);
         }
-        {   // end marker
-            const int slot = seq % kNS;
-            if (seq >= kNS) wait_or_abort(bar(kBarEmpty + slot), (uint32_t)(seq / kNS - 1) & 1u);
-            if (lane == 0) {
-                s_hdr[slot].item = -1;
-                mbar_arrive(bar(kBarFull + slot));
-            }
-        }
+        TCTRACE_END(2);
+        if (lane == 0) { TCP_FLUSH(0); }
         if (lane == 0) {   // the last CTA to stop claiming rewinds the counters for the next launch
             __threadfence();
             const int done = atomicAdd(a.counters + 3, 1);
@@ -335,76 +413,201 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 __threadfence();
             }
         }
-    } else if (warp >= kMmaWarp) {
+    } else if (warp >= kVWarp && warp < kVWarp + 3) {
+        // ------------------------------ follower producers ------------------------------
+        // Warp 12: V of the even slots, 13: K of the odd slots, 14: V of the odd slots.  Each follows
+        // the item ring and issues its share (one warp cannot issue TMA copies fast enough for more).
+        const bool is_v = warp != kVWarp + 1;
+        const int par = warp == kVWarp ? 0 : 1;
+        const int nring = is_v ? kNV : kNK;
+        const int bfull = is_v ? kBarFullV : kBarFullK, bempty = is_v ? kBarEmptyV : kBarEmptyK;
+        const uint32_t ring = sbase + (is_v ? kVOff : 0);
+        const CUtensorMap* tm = is_v ? &tm_v : &tm_k;
+        int seq = 0;
+        for (int k = 0; !*s_abort; ++k) {
+            const int e = k % kNI;
+            wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u);
+            if (*s_abort) break;
+            const int item = s_item[e].item;
+            const int page_begin = s_item[e].it.page_begin, num_pages = s_item[e].it.num_pages;
+            const int kvh = s_item[e].it.kv_head;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarItemEmpty + e));
+            if (item < 0) break;
+            auto fetch_ids = [&](int first) {
+                return (first + lane < num_pages) ? __ldg(a.plan.seg_blocks + page_begin + first + lane) : 0;
+            };
+            const int ngroups = (num_pages + 3) / 4;
+            int ids = fetch_ids(0), ids_ahead = 0;
+            for (int g = 0; g < ngroups; ++g, ++seq) {
+                const int slot = seq % nring;
+                const int npg = min(4, num_pages - g * 4);
+                if ((g & 7) == 0) ids_ahead = fetch_ids((g + 8) * 4);
+                const int page = __shfl_sync(0xffffffffu, ids, (g & 7) * 4 + ((lane >> 1) & 3));   // lane = 2 * page + half
+                if ((g & 7) == 7) ids = ids_ahead;
+                if ((seq & 1) != par) continue;
+                if (seq >= nring) wait_or_abort(bar(bempty + slot), (uint32_t)(seq / nring - 1) & 1u);
+                if (*s_abort) break;
+                const uint32_t full = bar(bfull + slot);
+                if (lane == 0) mbar_arrive_expect_tx(full, npg * (kBlock * HD * 2));
+                __syncwarp();
+                if (lane < npg * 2) {
+                    const int y = (page * a.Hkv + kvh) * kBlock;
+                    tma_load_2d(ring + slot * kKBytes + (lane >> 1) * 2048 + (lane & 1) * 8192, tm, (lane & 1) * 64, y, full);
+                }
+            }
+        }
+    } else if (warp == kQWarp) {
+        // ------------------------------------ Q loader ------------------------------------
+        // Row r of the tile <-> (sharer r / G, head r % G of the item's KV head).  16-byte chunk c of a
+        // row goes to half c / 8, at chunk (c % 8) ^ (r % 8) of the row's 128 bytes (the 128-byte
+        // swizzle the MMA's shared-memory descriptor expects).
+        const int G = a.G;
+        for (int k = 0; !*s_abort; ++k) {
+            const int e = k % kNI;
+            wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u);
+            if (*s_abort) break;
+            const int item = s_item[e].item;
+            const WorkItem it = s_item[e].it;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarItemEmpty + e));
+            if (item < 0) break;
+            const int rows = it.num_sharers * G;
+            // the sharers of this lane's four rows, fetched before the wait below
+            Sharer sh[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = lane + 32 * i;
+                sh[i] = Sharer{};
+                if (r < rows) sh[i] = a.plan.sharers[it.sharer_begin + r / G];
+            }
+            // this Q tile is free once every Q K^T of the item before the previous one has completed
+            // and the softmax warps have read that item's row bases
+            if (k >= 2) wait_or_abort(bar(kBarQEmpty + (k & 1)), (uint32_t)((k >> 1) - 1) & 1u);
+            if (*s_abort) break;
+            const uint32_t qdst = sbase + kQOff + (k & 1) * kQBytes;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = lane + 32 * i;
+                const uint32_t rowdst = qdst + r * 128;
+                if (r < rows) {
+                    const int h = it.kv_head * G + r % G;
+                    s_rowbase[(k & 1) * 128 + r] = sh[i].mass_base + (int64_t)h * sh[i].nblk + it.seg_page_begin;
+                    const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) +
+                                                                      ((size_t)sh[i].branch * a.Hq + h) * HD);
+#pragma unroll
+                    for (int c = 0; c < 16; ++c)
+                        cp_async16(rowdst + (c >> 3) * 16384 + (((c & 7) ^ (r & 7)) << 4), src + c);
+                } else {
+                    s_rowbase[(k & 1) * 128 + r] = 0;
+#pragma unroll
+                    for (int c = 0; c < 16; ++c)
+                        *reinterpret_cast<uint4*>(smem + kQOff + (k & 1) * kQBytes + r * 128 + (c >> 3) * 16384 + (c & 7) * 16) =
+                            make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> the MMA's reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarQFull + (k & 1)));
+        }
+    } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
         // ------------------------- MMA issuers: warp 9 for warpgroup 0, warp 10 for warpgroup 1 -------------------------
-        // Each walks every slot header (to see item boundaries) and issues the MMAs of its own
-        // warpgroup's slots: S of the next own slot goes out before P V of the previous one, so S
-        // is ready by the time the warpgroup finishes its softmax.
+        // Slot number seq (counted over all items of the CTA) belongs to warpgroup seq % 2.  Each issuer
+        // walks every slot (observing each "landed" phase in order) and issues the MMAs of its own: S of
+        // own slot c goes into buffer c % 2 - free, because P V of own slot c - 2, which read P from
+        // it, was issued earlier by this same thread and the tensor pipe runs in order - and only then
+        // P V of own slot c - 1, once its P is there.
         if (lane == 0) {
             constexpr uint32_t kIdescQK = instr_desc(kSlotTokens, 0);
             constexpr uint32_t kIdescPV = instr_desc(HD, 1);
             const int wg = warp - kMmaWarp;
-            int c = 0;                   // own slots issued (all items)
-            bool first_pv = true;
-            int item_k = -1;
-            int pend_slot = -1, pend_npg = 0, pend_c = 0;
-            TCPROF_DECL;
+            const uint32_t qbase0 = sbase + kQOff;
+            int seq = 0;                 // slots seen (all items, both warpgroups)
+            int c = 0;                   // own slots issued
+            int pend_slot = -1, pend_seq = 0, pend_npg = 0, pend_c = 0, pend_item = 0;
+            bool pend_first = false;
+            TCP_DECL;
+            TCTRACE_DECL(wg);
             auto flush_pv = [&]() {
                 if (pend_slot < 0) return;
-                TCPROF_WAIT(3, wait_or_abort(bar(kBarPFull + wg), (uint32_t)pend_c & 1u));
+                TCTRACE(2048 + (pend_seq & 1023));
+                TCP_WAIT(1, wait_or_abort(bar(kBarPFull + wg * 2 + (pend_c & 1)), (uint32_t)(pend_c >> 1) & 1u));
+                TCTRACE(3072 + (pend_seq & 1023));
+                // the first P V of an item overwrites O: both warpgroups must have read out the previous item
+                if (pend_first && pend_item > 0) TCP_WAIT(2, wait_or_abort(bar(kBarEpiB), (uint32_t)(pend_item - 1) & 1u));
+                TCP_WAIT(5, wait_or_abort(bar(kBarFullV + pend_slot), (uint32_t)(pend_seq / kNV) & 1u));
+                TCTRACE(3072 + 512 + (pend_seq & 511));
                 if (!*s_abort) {
                     tc_fence_after();
-                    const uint32_t vbase = sbase + pend_slot * kSlotBytes + kKBytes;
-                    TCPROF_WAIT(6, for (int j = 0; j < pend_npg; ++j) {
+                    const uint32_t vbase = sbase + kVOff + pend_slot * kKBytes;
+                    const uint32_t pcol = tmem + kColS + (uint32_t)(wg * 2 + (pend_c & 1)) * 64;
+                    TCP_WAIT(7, for (int j = 0; j < pend_npg; ++j) {
                         const uint64_t bd = smem_desc(vbase + j * 2048, 8192, 1024);
-                        umma_ts(tmem + kColO + wg * 128, tmem + kColP + wg * 32 + j * 8, bd, kIdescPV,
-                                (first_pv && j == 0) ? 0u : 1u);
-                    });
-                    first_pv = false;
-                    TCPROF_WAIT(7, tc_commit(bar(kBarODone + wg));
-                    tc_commit(bar(kBarEmpty + pend_slot)));
+                        umma_ts(tmem + kColO + wg * 128, pcol + j * 8, bd, kIdescPV, (pend_first && j == 0) ? 0u : 1u);
+                    }
+                    tc_commit(bar(kBarODone + wg));
+                    tc_commit(bar(kBarEmptyV + pend_slot)));
                 }
                 pend_slot = -1;
             };
-            for (int seq = 0; !*s_abort; ++seq) {
-                const int slot = seq % kNS;
-                TCPROF_WAIT(1, wait_or_abort(bar(kBarFull + slot), (uint32_t)(seq / kNS) & 1u));
+            for (int k = 0; !*s_abort; ++k) {
+                const int e = k % kNI;
+                TCP_WAIT(3, wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u));
                 if (*s_abort) break;
-                const int4 hdr = *reinterpret_cast<const int4*>(&s_hdr[slot]);   // item, group, pages, last
-                if (hdr.x < 0) break;
-                const int g = hdr.y, npg = hdr.z;
-                const bool own = (g & 1) == wg;
-                // a slot of the other warpgroup is only looked at: hand the header back
-                if (!own) mbar_arrive(bar(kBarEmpty + slot));
-                if (g == 0) {
-                    flush_pv();
-                    ++item_k;
-                    TCPROF_WAIT(4, wait_or_abort(bar(kBarQFull), (uint32_t)item_k & 1u));
+                const int item = s_item[e].item;
+                const int ngroups = s_item[e].num_groups;
+                const int num_pages = s_item[e].it.num_pages;
+                mbar_arrive(bar(kBarItemEmpty + e));
+                if (item < 0) break;
+                TCP_WAIT(4, wait_or_abort(bar(kBarQFull + (k & 1)), (uint32_t)(k >> 1) & 1u));
+                if (*s_abort) break;
+                bool first_own = true;
+                const uint32_t qbase = qbase0 + (k & 1) * kQBytes;
+                for (int g = 0; g < ngroups; ++g, ++seq) {
+                    if ((seq & 1) != wg) continue;   // ring sizes are even: a slot's every phase is this warpgroup's or never
+                    const int slot = seq % kNK;
+                    TCTRACE(1024 + (seq & 1023));
+                    TCP_WAIT(5, wait_or_abort(bar(kBarFullK + slot), (uint32_t)(seq / kNK) & 1u));
                     if (*s_abort) break;
-                    first_pv = true;
+                    TCTRACE(seq & 1023);
+#ifdef EXP_PVFIRST
+                    flush_pv();
+#endif
+                    tc_fence_after();
+                    const uint32_t kbase = sbase + slot * kKBytes;
+                    const uint32_t scol = tmem + kColS + (uint32_t)(wg * 2 + (c & 1)) * 64;
+                    TCP_WAIT(6, for (int ks = 0; ks < HD / 16; ++ks) {
+                        const uint64_t ad = smem_desc(qbase + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
+                        const uint64_t bd = smem_desc(kbase + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
+                        umma_ss(scol, ad, bd, kIdescQK, ks > 0 ? 1u : 0u);
+                    }
+                    tc_commit(bar(kBarSFull + wg * 2 + (c & 1)));
+                    tc_commit(bar(kBarEmptyK + slot)));   // K of the slot is free as soon as S is there
+                    flush_pv();   // P V of the previous own slot, after S of this one
+                    pend_slot = seq % kNV;
+                    pend_seq = seq;
+                    pend_npg = min(4, num_pages - g * 4);
+                    pend_c = c;
+                    pend_item = k;
+                    pend_first = first_own;
+                    first_own = false;
+                    ++c;
                 }
-                if (!own) continue;
-                if (c > 0) TCPROF_WAIT(2, wait_or_abort(bar(kBarSFree + wg), (uint32_t)(c - 1) & 1u));
                 if (*s_abort) break;
-                tc_fence_after();
-                const uint32_t kbase = sbase + slot * kSlotBytes;
-                TCPROF_WAIT(5, for (int ks = 0; ks < HD / 16; ++ks) {
-                    const uint64_t bd = smem_desc(kbase + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
-                    umma_ts(tmem + kColS + wg * 64, tmem + kColQ + ks * 8, bd, kIdescQK, ks > 0 ? 1u : 0u);
-                });
-                tc_commit(bar(kBarSFull + wg));
-                mbar_arrive(bar(kBarEmpty + slot));   // this issuer's share of the slot's release (the P V commit is another)
-                flush_pv();   // P V of the previous own slot, after S of this one
-                pend_slot = slot;
-                pend_npg = npg;
-                pend_c = c;
-                ++c;
+                tc_commit(bar(kBarQEmpty + (k & 1)));   // this issuer's Q K^T of the item (if any) have completed
+                // the item's last P V goes out now rather than after the next item's first S: the
+                // warpgroups' epilogue waits for it
+                flush_pv();
             }
             flush_pv();
-            if (wg == 0) { TCPROF_FLUSH(0); }
+            TCTRACE_END(wg);
+            TCP_FLUSH(8 + 8 * wg);
         }
         __syncwarp();
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 192;" ::: "memory");
         // ------------------------------------ softmax warps ------------------------------------
         const int wg = warp >> 2, quad = warp & 3;
         const int row = quad * 32 + lane;
@@ -413,96 +616,62 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const int G = a.G;
         float2* s_ml = reinterpret_cast<float2*>(smem + kMlOff);
 
-        int cwg = 0;        // slots this warpgroup has processed (all items)
-        int citem = 0;      // ... in the current item
-        int item_k = -1;
-        WorkItem it{};
-        int rows = 0;
-        bool valid = false, warp_has_rows = false;
-        int64_t mb = 0;
-        float m = -INFINITY, l = 0.f;
-        TCPROF_DECL;
+        int seq = 0;        // slots seen (all items, both warpgroups)
+        int c = 0;          // own slots processed (all items)
+        TCP_DECL;
 #ifdef RKSC_WAIT_PROFILE
-        unsigned long long tcq[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        long long tcq_t = 0;
+        int tr_n = 0; const bool tr_on = blockIdx.x == 0 && threadIdx.x == 0; long long* const tr_buf = g_tc_trace[3];
 #endif
 
-        for (int seq = 0;; ++seq) {
-            const int slot = seq % kNS;
-            TCPROF_WAIT(1, wait_or_abort(bar(kBarFull + slot), (uint32_t)(seq / kNS) & 1u));
+        for (int k = 0; !*s_abort; ++k) {
+            const int e = k % kNI;
+            TCP_WAIT(1, wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u));
             if (*s_abort) break;
-            const int4 hdr = *reinterpret_cast<const int4*>(&s_hdr[slot]);   // item, group, pages, last
-            if (hdr.x < 0) break;
-            const int g = hdr.y, npg = hdr.z;
-            int ngroups = 0;
-            if (g == 0) {
-                it = s_hdr[slot].it;
-            }
-            ngroups = s_hdr[slot].num_groups;
+            const int item = s_item[e].item;
+            const int ngroups = s_item[e].num_groups;
+            const int it_num_tokens = s_item[e].it.num_tokens, it_num_pages = s_item[e].it.num_pages;
+            const int it_part_row_base = s_item[e].it.part_row_base;
+            const int rows = s_item[e].it.num_sharers * G;
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarEmpty + slot));   // header read
+            if (lane == 0) mbar_arrive(bar(kBarItemEmpty + e));
+            if (item < 0) break;
+            // row bases of the item (written by the Q loader before it signals the Q tile)
+            TCP_WAIT(2, wait_or_abort(bar(kBarQFull + (k & 1)), (uint32_t)(k >> 1) & 1u));
+            if (*s_abort) break;
+            const bool valid = row < rows;
+            const bool warp_has_rows = quad * 32 < rows;
+            const int64_t mb = s_rowbase[(k & 1) * 128 + row];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarQEmpty + (k & 1)));   // row bases read
+            float m = -INFINITY, l = 0.f;
+            int citem = 0;      // own slots of this item
 
-            if (g == 0) {
-                // ---- new item: row bookkeeping and the Q tile ----
-                ++item_k;
-                rows = it.num_sharers * G;
-                valid = row < rows;
-                warp_has_rows = quad * 32 < rows;
-                m = -INFINITY;
-                l = 0.f;
-                citem = 0;
-                const uint4* qsrc = nullptr;
-                if (valid) {
-                    const Sharer sh = a.plan.sharers[it.sharer_begin + row / G];
-                    const int h = it.kv_head * G + row % G;
-                    mb = sh.mass_base + (int64_t)h * sh.nblk + it.seg_page_begin;
-                    qsrc = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) +
-                                                          ((size_t)sh.branch * a.Hq + h) * HD + wg * 64);
-                }
-                // this warpgroup stages half `wg` (64 of the 128 dims) of every row into the Q columns of
-                // tensor memory: thread = row = TMEM lane, two bf16 per 32-bit column (A operand of Q K^T)
-                {
-                    uint32_t qr[32];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                        if (valid) v = __ldg(qsrc + c);
-                        qr[4 * c] = v.x;
-                        qr[4 * c + 1] = v.y;
-                        qr[4 * c + 2] = v.z;
-                        qr[4 * c + 3] = v.w;
-                    }
-                    tmem_st32(lane_addr + kColQ + wg * 32, qr);
-                    tmem_wait_st();
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarQFull));
-            }
-
-            if ((g & 1) == wg) {
+            for (int g = 0; g < ngroups; ++g, ++seq) {
+                if ((seq & 1) != wg) continue;
                 // ---- this warpgroup's slot: S row -> softmax -> P row ----
-                TCPROF_WAIT(2, wait_or_abort(bar(kBarSFull + wg), (uint32_t)cwg & 1u));
+                const uint32_t scol = lane_addr + kColS + (uint32_t)(wg * 2 + (c & 1)) * 64;
+                TCTRACE(5);
+                TCP_WAIT(3, wait_or_abort(bar(kBarSFull + wg * 2 + (c & 1)), (uint32_t)(c >> 1) & 1u));
                 if (*s_abort) break;
                 tc_fence_after();
-#ifdef RKSC_WAIT_PROFILE
-                tcq_t = clock64();
-#endif
+                TCTRACE(6);
                 uint32_t sr[2][32];
-                tmem_ld32(lane_addr + kColS + wg * 64, sr[0]);
-                tmem_ld32(lane_addr + kColS + wg * 64 + 32, sr[1]);
+#ifdef EXP_STREAMONLY
+                for (int j = 0; j < 64; ++j) sr[j >> 5][j & 31] = 0u;
+                if (c >= 0) { __syncwarp(); if (lane == 0) mbar_arrive(bar(kBarPFull + wg * 2 + (c & 1))); ++c; ++citem; continue; }
+#endif
+                tmem_ld32(scol, sr[0]);
+                tmem_ld32(scol + 32, sr[1]);
                 tmem_wait_ld();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarSFree + wg));
-                TCPROF_MARK(0);
 
-                const int nvalid = it.num_tokens - g * kSlotTokens;   // tokens of this slot that exist
+                const int nvalid = it_num_tokens - g * kSlotTokens;   // tokens of this slot that exist
+                const int npg = min(4, it_num_pages - g * 4);
                 float mx = -INFINITY;
-#ifdef RKSC_TC_SKIP_SOFTMAX
-                mx = __uint_as_float(sr[0][0]) * 0.f;
+#ifdef EXP_NOMAX
+                if (false) {
 #else
                 if (warp_has_rows) {
+#endif
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
                     if (nvalid >= kSlotTokens) {
 #pragma unroll
@@ -522,8 +691,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     }
                     mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 }
-#endif
-                TCPROF_MARK(1);
 
                 // Running maximum with slack: m is raised (and O, l rescaled) only when a row's maximum
                 // moved up by more than kRescaleStep, so p = 2^(s - m) stays below 2^kRescaleStep and the
@@ -531,43 +698,54 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (citem == 0) {
                     if (valid) m = mx;
                 } else {
-                    // the previous P V of this warpgroup must be complete before P is overwritten or O touched
-                    TCPROF_WAIT(3, wait_or_abort(bar(kBarODone + wg), (uint32_t)(cwg - 1) & 1u));
-                    if (*s_abort) break;
-                    tc_fence_after();
                     const bool grew = valid && (mx > m + kRescaleStep);
                     if (__any_sync(0xffffffffu, grew)) {
+                        // O must be at rest: P V of this warpgroup's previous slot has to be complete
+                        wait_or_abort(bar(kBarODone + wg), (uint32_t)(c - 1) & 1u);
+                        if (*s_abort) break;
+                        tc_fence_after();
                         const float alpha = grew ? fast_exp2(m - mx) : 1.f;
                         l *= alpha;
 #pragma unroll 1
-                        for (int c = 0; c < HD / 32; ++c) {
+                        for (int cc = 0; cc < HD / 32; ++cc) {
                             uint32_t o[32];
-                            tmem_ld32(lane_addr + kColO + wg * 128 + c * 32, o);
+                            tmem_ld32(lane_addr + kColO + wg * 128 + cc * 32, o);
                             tmem_wait_ld();
 #pragma unroll
                             for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-                            tmem_st32(lane_addr + kColO + wg * 128 + c * 32, o);
+                            tmem_st32(lane_addr + kColO + wg * 128 + cc * 32, o);
                         }
                         tmem_wait_st();
                         if (grew) m = mx;
                     }
                 }
-                TCPROF_MARK(2);
 
+                // p = 2^(s - m), its per-page sums, and the P row as bf16 pairs (A operand of P V)
                 float ps[4] = {0.f, 0.f, 0.f, 0.f};
-#ifndef RKSC_TC_SKIP_SOFTMAX
+                uint32_t pk[32];
                 if (warp_has_rows) {
-                    const float mm = valid ? m : 0.f;   // rows past the item's end hold zeros: harmless, never read
+                    const float mm = valid ? m : 0.f;   // rows past the item's end: harmless, never read
 #pragma unroll
-                    for (int j = 0; j < 64; ++j) {
-                        const float p = fast_exp2(__uint_as_float(sr[j >> 5][j & 31]) - mm);
-                        sr[j >> 5][j & 31] = __float_as_uint(p);
-                        ps[j >> 4] += p;
+                    for (int j = 0; j < 32; ++j) {
+#ifdef EXP_NOEXP
+                        const float p0 = (__uint_as_float(sr[(2 * j) >> 5][(2 * j) & 31]) - mm) * 0.001f;
+                        const float p1 = (__uint_as_float(sr[(2 * j + 1) >> 5][(2 * j + 1) & 31]) - mm) * 0.001f;
+#else
+                        const float p0 = fast_exp2(__uint_as_float(sr[(2 * j) >> 5][(2 * j) & 31]) - mm);
+                        const float p1 = fast_exp2(__uint_as_float(sr[(2 * j + 1) >> 5][(2 * j + 1) & 31]) - mm);
+#endif
+                        ps[j >> 3] += p0;
+                        ps[j >> 3] += p1;
+                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+                        pk[j] = *reinterpret_cast<const uint32_t*>(&b2);
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 64; ++j) sr[j >> 5][j & 31] = 0u;
+                    for (int j = 0; j < 32; ++j) pk[j] = 0u;
                 }
+                // over the first 32 columns of the S buffer, whose 64 values are all in registers by now
+#ifndef EXP_NOPST
+                tmem_st32(scol, pk);
 #endif
                 l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
                 if (valid && a.block_mass != nullptr) {
@@ -575,91 +753,76 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     for (int j = 0; j < 4; ++j)
                         if (j < npg) a.block_mass[mb + g * 4 + j] = m + fast_log2(ps[j]);
                 }
-                TCPROF_MARK(3);
-                // P row as bf16 pairs into this warpgroup's P columns of tensor memory (A operand of P V)
-                {
-                    uint32_t pk[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(sr[(2 * j) >> 5][(2 * j) & 31]),
-                                                                        __uint_as_float(sr[(2 * j + 1) >> 5][(2 * j + 1) & 31]));
-                        pk[j] = *reinterpret_cast<const uint32_t*>(&b2);
-                    }
-                    tmem_st32(lane_addr + kColP + wg * 32, pk);
-                    tmem_wait_st();
-                }
+                tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPFull + wg));
-                TCPROF_MARK(4);
-                ++cwg;
+                if (lane == 0) mbar_arrive(bar(kBarPFull + wg * 2 + (c & 1)));
+                TCTRACE(7);
+                ++c;
                 ++citem;
             }
-
-            if (!hdr.w) continue;
+            if (*s_abort) break;
 
             // ---- item epilogue: merge the two warpgroups' states, write the partial ----
-            if (citem > 0) {
-                wait_or_abort(bar(kBarODone + wg), (uint32_t)(cwg - 1) & 1u);
+            TCTRACE(1);
+            const bool have_self = citem > 0;                 // warpgroup-uniform
+            const bool have_oth = ngroups - citem > 0;        // the other warpgroup had a slot
+            if (have_self) {
+                TCP_WAIT(4, wait_or_abort(bar(kBarODone + wg), (uint32_t)(c - 1) & 1u));
                 if (*s_abort) break;
                 tc_fence_after();
             }
-            s_ml[wg * 128 + row] = make_float2(m, l);
+            TCTRACE(2);
+            s_ml[((k & 1) * 2 + wg) * 128 + row] = make_float2(m, l);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarEpiA));
-            TCPROF_WAIT(4, wait_or_abort(bar(kBarEpiA), (uint32_t)item_k & 1u));
+            TCP_WAIT(5, wait_or_abort(bar(kBarEpiA), (uint32_t)k & 1u));
             if (*s_abort) break;
             tc_fence_after();
+            TCTRACE(3);
             {
-                const float2 oth = s_ml[(1 - wg) * 128 + row];
-                const bool have_self = citem > 0;                       // warpgroup-uniform
-                const bool have_oth = ngroups > (1 - wg);               // the other warpgroup had a slot
+                const float2 oth = s_ml[((k & 1) * 2 + (1 - wg)) * 128 + row];
                 const float M = fmaxf(have_self ? m : -INFINITY, have_oth ? oth.x : -INFINITY);
                 const float w_self = have_self ? fast_exp2(m - M) : 0.f;
                 const float w_oth = have_oth ? fast_exp2(oth.x - M) : 0.f;
                 const float L = w_self * l + w_oth * oth.y;
                 const float inv = 1.f / L;
                 const float c_self = w_self * inv, c_oth = w_oth * inv;
-                float* dst = a.part_o + ((size_t)it.part_row_base + row) * HD + wg * 64;
+                float* dst = a.part_o + ((size_t)it_part_row_base + row) * HD + wg * 64;
 #pragma unroll 1
-                for (int hh = 0; hh < 2; ++hh) {
-                    float acc[32];
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t os[16], oo[16];
+                    if (have_self) tmem_ld16(lane_addr + kColO + wg * 128 + wg * 64 + q4 * 16, os);
+                    if (have_oth) tmem_ld16(lane_addr + kColO + (1 - wg) * 128 + wg * 64 + q4 * 16, oo);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-                    if (have_self) {
-                        uint32_t o[32];
-                        tmem_ld32(lane_addr + kColO + wg * 128 + wg * 64 + hh * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) acc[j] = c_self * __uint_as_float(o[j]);
+                    for (int j = 0; j < 16; ++j) {
+                        float v = 0.f;
+                        if (have_self) v = c_self * __uint_as_float(os[j]);
+                        if (have_oth) v += c_oth * __uint_as_float(oo[j]);
+                        os[j] = __float_as_uint(v);
                     }
-                    if (have_oth) {
-                        uint32_t o[32];
-                        tmem_ld32(lane_addr + kColO + (1 - wg) * 128 + wg * 64 + hh * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) acc[j] += c_oth * __uint_as_float(o[j]);
-                    }
+#ifdef EXP_NOEPIST
+                    if (valid && os[3] == 0x12345u) {
+#else
                     if (valid) {
+#endif
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            *reinterpret_cast<float4*>(dst + hh * 32 + j * 4) =
-                                make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+                        for (int j = 0; j < 4; ++j)
+                            *reinterpret_cast<uint4*>(dst + q4 * 16 + j * 4) =
+                                make_uint4(os[4 * j], os[4 * j + 1], os[4 * j + 2], os[4 * j + 3]);
                     }
                 }
-                if (valid && wg == 0) a.part_lse[(size_t)it.part_row_base + row] = M + fast_log2(L);
+                if (valid && wg == 0) a.part_lse[(size_t)it_part_row_base + row] = M + fast_log2(L);
             }
+            TCTRACE(4);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarEpiB));
-            TCPROF_WAIT(5, wait_or_abort(bar(kBarEpiB), (uint32_t)item_k & 1u));
-            if (*s_abort) break;
+            if (lane == 0) mbar_arrive(bar(kBarEpiB));   // the issuers wait for this before the next item's first P V
         }
 #ifdef RKSC_WAIT_PROFILE
-        if (warp == 0 && lane == 0) {
-            tcp[6] = (unsigned long long)cwg; tcp[7] = (unsigned long long)(item_k + 1); TCPROF_FLUSH(8);
-            for (int _i = 0; _i < 8; ++_i) g_tc_prof[blockIdx.x + 128][_i] = tcq[_i];
-        }
+        if (tr_on) g_tc_trace_n[3] = tr_n;
+        if (wg == 0 && quad == 0 && lane == 0) { tcp[6] = (unsigned long long)c; TCP_FLUSH(24); }
 #endif
     }
 
@@ -675,6 +838,13 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 }  // namespace
 
 #ifdef RKSC_WAIT_PROFILE
+extern "C" __attribute__((visibility("default"))) int rksc_debug_tc_trace(long long* host_out, int* n) {
+    if (cudaMemcpyFromSymbol(n, g_tc_trace_n, sizeof(g_tc_trace_n)) != cudaSuccess) return -1;
+    return cudaMemcpyFromSymbol(host_out, g_tc_trace, sizeof(g_tc_trace)) == cudaSuccess ? 0 : -1;
+}
+extern "C" __attribute__((visibility("default"))) int rksc_debug_tc_dbg(int* host_out) {
+    return cudaMemcpyFromSymbol(host_out, g_tc_dbg, sizeof(g_tc_dbg)) == cudaSuccess ? 0 : -1;
+}
 extern "C" __attribute__((visibility("default"))) int rksc_debug_tc_profile(unsigned long long* host_out) {
     return cudaMemcpyFromSymbol(host_out, g_tc_prof, sizeof(g_tc_prof)) == cudaSuccess ? 0 : -1;
 }
