@@ -160,9 +160,10 @@ struct SmemLayout {
     static constexpr int kScrOff = kRing;
     static constexpr int kMlOff = kScrOff + kCW * kScrWarp;   // m[4][16], l[4][16]
     static constexpr int kBarOff = kMlOff + 2 * kCW * 16 * 4;  // full[kNS], empty[kNS]
-    static constexpr int kHdrOff = kBarOff + ((2 * kNS * 8 + 8 + 15) / 16) * 16;  // after the barriers (+ the consumers' own)
+    static constexpr int kHdrOff = kBarOff + ((3 * kNS * 8 + 8 + 15) / 16) * 16;  // after the barriers: full, empty, consumers' own, header ready
     static_assert(kBarOff % 8 == 0 && kHdrOff % 16 == 0 && kScrOff % 16 == 0, "shared-memory alignment");
-    static constexpr int kFlagOff = kHdrOff + kNS * 64;        // one SlotHeader per slot
+    static constexpr int kPagesOff = kHdrOff + kNS * 64;       // one SlotHeader per slot, then its page ids
+    static constexpr int kFlagOff = kPagesOff + kNS * kSP * 4;
     // an item with <= 8 rows merges its four page lanes through the sub-page regions of its last slot
     static_assert(8 * (HD + 4) * 4 + 64 <= kPage, "small-row merge scratch must fit in a sub-page");
     static constexpr int kTotal = kFlagOff + 16;
@@ -181,14 +182,17 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     const uint32_t bar_full = ring + SL::kBarOff;
     const uint32_t bar_empty = bar_full + kNS * 8;
     const uint32_t bar_cons = bar_empty + kNS * 8;   // the four consumer warps meet here in the item epilogue
+    const uint32_t bar_hdr = bar_cons + 8;           // [kNS] header and page ids of the slot written (K producer -> V producer)
     SlotHeader* s_hdr = reinterpret_cast<SlotHeader*>(smem + SL::kHdrOff);
+    int32_t* s_pages = reinterpret_cast<int32_t*>(smem + SL::kPagesOff);
     volatile int32_t* s_abort = reinterpret_cast<volatile int32_t*>(smem + SL::kFlagOff);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         for (int i = 0; i < kNS; ++i) {
-            mbar_init(bar_full + 8 * i, 1);
+            mbar_init(bar_full + 8 * i, 2);     // the K and the V producer
             mbar_init(bar_empty + 8 * i, kCW);
+            mbar_init(bar_hdr + 8 * i, 1);
         }
         mbar_init(bar_cons, kCW);
         *s_abort = 0;
@@ -256,17 +260,19 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     h.it = it;
                     h.pad[0] = h.pad[1] = 0;
                     s_hdr[slot] = h;
-                    mbar_arrive_expect_tx(bar, npg * SL::kPage);
+                }
+                if (lane < kSP) s_pages[slot * kSP + lane] = page;
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar_hdr + 8 * slot);                 // the V producer may follow
+                    mbar_arrive_expect_tx(bar, npg * SL::kTile);     // this warp's half of the slot: K
                 }
                 __syncwarp();
                 if (lane < npg) {
                     const int y = (page * a.Hkv + it.kv_head) * kBlock;
                     const uint32_t dst = ring + slot * SL::kSlot + lane * SL::kPage;
 #pragma unroll
-                    for (int hh = 0; hh < HD / 64; ++hh) {
-                        tma_load_2d(dst + hh * 2048, &tm_k, hh * 64, y, bar);
-                        tma_load_2d(dst + SL::kTile + hh * 2048, &tm_v, hh * 64, y, bar);
-                    }
+                    for (int hh = 0; hh < HD / 64; ++hh) tma_load_2d(dst + hh * 2048, &tm_k, hh * 64, y, bar);
                 }
             }
             idx = nidx;
@@ -282,6 +288,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             if (seq >= kNS) wait_or_abort(bar_empty + 8 * slot, (uint32_t)(seq / kNS - 1) & 1u);
             if (lane == 0) {
                 s_hdr[slot].item = -1;
+                mbar_arrive(bar_hdr + 8 * slot);
                 mbar_arrive(bar_full + 8 * slot);
             }
         }
@@ -298,6 +305,37 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         // When this grid was launched behind the tcgen05 kernel without waiting for it, it must not
         // complete before that kernel has: the merge kernel waits on this grid only.
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
+
+    if (warp == kCW + 1) {
+        // ------------------------------ V producer warp ------------------------------
+        // One warp cannot issue TMA copies fast enough for a CTA's share of the memory bandwidth: this
+        // one follows the K producer slot by slot (header and page ids through shared memory) and
+        // issues the V half of every slot.
+        for (int seq = 0; !*s_abort; ++seq) {
+            const int slot = seq % kNS;
+            wait_or_abort(bar_hdr + 8 * slot, (uint32_t)(seq / kNS) & 1u);
+            if (*s_abort) break;
+            const int item = s_hdr[slot].item;
+            const uint32_t bar = bar_full + 8 * slot;
+            if (item < 0) {
+                if (lane == 0) mbar_arrive(bar);
+                break;
+            }
+            const int npg = s_hdr[slot].num_pages;
+            const int kvh = s_hdr[slot].it.kv_head;
+            const int page = s_pages[slot * kSP + (lane & (kSP - 1))];
+            __syncwarp();
+            if (lane == 0) mbar_arrive_expect_tx(bar, npg * SL::kTile);
+            __syncwarp();
+            if (lane < npg) {
+                const int y = (page * a.Hkv + kvh) * kBlock;
+                const uint32_t dst = ring + slot * SL::kSlot + lane * SL::kPage + SL::kTile;
+#pragma unroll
+                for (int hh = 0; hh < HD / 64; ++hh) tma_load_2d(dst + hh * 2048, &tm_v, hh * 64, y, bar);
+            }
+        }
         return;
     }
 

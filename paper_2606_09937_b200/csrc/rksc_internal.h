@@ -15,7 +15,7 @@ constexpr int kTcMinRows = 17;              // from this many stacked rows on, t
 constexpr int kTcMaxRows = 128;             // rows of one tcgen05 work item (the MMA's M)
 constexpr int kMaxPagesPerItem = 512;       // page ids a CTA caches in shared memory
 constexpr int kConsumerWarps = 4;           // MMA warps of the segment kernel
-constexpr int kWarpKernelThreads = (kConsumerWarps + 1) * 32;   // + one TMA producer warp
+constexpr int kWarpKernelThreads = (kConsumerWarps + 2) * 32;   // + two TMA producer warps (K, V)
 constexpr int kSubPages = 4;                // pages staged per ring slot
 constexpr int kRingSlots = 3;               // ring slots per CTA
 constexpr int kCtasPerSm = 2;               // persistent CTAs per SM
