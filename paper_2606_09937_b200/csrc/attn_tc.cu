@@ -39,9 +39,10 @@ namespace {
 constexpr int HD = 128;
 constexpr int kSmWarps = 8;                       // softmax warps (two warpgroups)
 constexpr int kProducerWarp = kSmWarps;           // 8
-constexpr int kMmaWarp = kSmWarps + 1;            // 9 and 10: MMA issuers of warpgroup 0 and 1
+constexpr int kMmaWarp = kSmWarps + 1;            // 9 and 10: Q K^T issuers of warpgroup 0 and 1
 constexpr int kQWarp = kSmWarps + 3;              // 11: Q loader
-constexpr int kVWarp = kSmWarps + 4;              // 12, 13, 14: follower producers (V even slots, K odd, V odd)
+constexpr int kVWarp = kSmWarps + 4;              // 12: V producer
+constexpr int kPvWarp = kSmWarps + 5;             // 13 and 14: P V issuers of warpgroup 0 and 1
 constexpr int kTcThreads = (kSmWarps + 8) * 32;   // 512: four warpgroups (warp 15 idles), so that registers can be re-divided
 constexpr int kNK = 4;                            // K ring slots (even: a slot always serves the same warpgroup)
 constexpr int kNV = 4;                            // V ring slots (even)
@@ -70,7 +71,8 @@ constexpr int kBarQEmpty = kBarQFull + 2;         // [2]    every Q K^T of the i
 constexpr int kBarSFull = kBarQEmpty + 2;         // [2][2] S of the warpgroup's slot is in its buffer
 constexpr int kBarPFull = kBarSFull + 4;          // [2][2] P of the slot is in the buffer
 constexpr int kBarODone = kBarPFull + 4;          // [2]    P V of the warpgroup's slot has completed
-constexpr int kBarEpiA = kBarODone + 2;           //        item epilogue: (m, l) published
+constexpr int kBarPVDone = kBarODone + 2;         // [2][2] ... per S buffer: the buffer may take the next S
+constexpr int kBarEpiA = kBarPVDone + 4;          //        item epilogue: (m, l) published
 constexpr int kBarEpiB = kBarEpiA + 1;            //        item epilogue: accumulators read
 constexpr int kNumBars = kBarEpiB + 1;
 constexpr int kItemOff = kBarOff + ((kNumBars * 8 + 15) / 16) * 16;
@@ -118,12 +120,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// The same with a suspend-time hint (nanoseconds): the thread sleeps in hardware until the phase
+// completes or the time is up, instead of spinning - a dozen helper warps polling in a tight loop
+// take issue slots from the softmax warps of their scheduler.
+__device__ __forceinline__ bool mbar_try_wait_sleep(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
 // Bounded wait: gives up after 2^32 SM cycles (about two seconds).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_sleep(bar, parity, 20000u)) return true;
         if (clock64() - t0 > (1ll << 32)) return false;
     }
 }
@@ -280,7 +298,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         }
         for (int i = 0; i < kNI; ++i) {
             mbar_init(bar(kBarItemFull + i), 1);
-            mbar_init(bar(kBarItemEmpty + i), kSmWarps + 6);   // 8 softmax warps, 2 issuers, Q loader, 3 follower producers
+            mbar_init(bar(kBarItemEmpty + i), kSmWarps + 6);   // 8 softmax warps, 4 issuers, Q loader, V producer
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(kBarQFull + i), 1);
@@ -292,6 +310,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         }
         mbar_init(bar(kBarODone + 0), 1);
         mbar_init(bar(kBarODone + 1), 1);
+        for (int i = 0; i < 4; ++i) mbar_init(bar(kBarPVDone + i), 1);
         mbar_init(bar(kBarEpiA), kSmWarps);
         mbar_init(bar(kBarEpiB), kSmWarps);
         *s_abort = 0;
@@ -385,7 +404,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 // lane = 2 * page + half
                 const int page = __shfl_sync(0xffffffffu, ids, (g & 7) * 4 + ((lane >> 1) & 3));
                 if ((g & 7) == 7) ids = ids_ahead;
-                if (seq & 1) continue;   // odd slots: warp 13
                 TCTRACE(1024 + (seq & 1023));
                 if (seq >= kNK) TCP_WAIT(1, wait_or_abort(bar(kBarEmptyK + kslot), (uint32_t)(seq / kNK - 1) & 1u));
                 if (*s_abort) break;
@@ -413,16 +431,14 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 __threadfence();
             }
         }
-    } else if (warp >= kVWarp && warp < kVWarp + 3) {
-        // ------------------------------ follower producers ------------------------------
-        // Warp 12: V of the even slots, 13: K of the odd slots, 14: V of the odd slots.  Each follows
-        // the item ring and issues its share (one warp cannot issue TMA copies fast enough for more).
-        const bool is_v = warp != kVWarp + 1;
-        const int par = warp == kVWarp ? 0 : 1;
-        const int nring = is_v ? kNV : kNK;
-        const int bfull = is_v ? kBarFullV : kBarFullK, bempty = is_v ? kBarEmptyV : kBarEmptyK;
-        const uint32_t ring = sbase + (is_v ? kVOff : 0);
-        const CUtensorMap* tm = is_v ? &tm_v : &tm_k;
+    } else if (warp == kVWarp) {
+        // ------------------------------ V producer ------------------------------
+        // Follows the item ring and streams the V half of every slot (one warp cannot issue TMA
+        // copies fast enough for both halves).
+        const int nring = kNV;
+        const int bfull = kBarFullV, bempty = kBarEmptyV;
+        const uint32_t ring = sbase + kVOff;
+        const CUtensorMap* tm = &tm_v;
         int seq = 0;
         for (int k = 0; !*s_abort; ++k) {
             const int e = k % kNI;
@@ -445,7 +461,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if ((g & 7) == 0) ids_ahead = fetch_ids((g + 8) * 4);
                 const int page = __shfl_sync(0xffffffffu, ids, (g & 7) * 4 + ((lane >> 1) & 3));   // lane = 2 * page + half
                 if ((g & 7) == 7) ids = ids_ahead;
-                if ((seq & 1) != par) continue;
                 if (seq >= nring) wait_or_abort(bar(bempty + slot), (uint32_t)(seq / nring - 1) & 1u);
                 if (*s_abort) break;
                 const uint32_t full = bar(bfull + slot);
@@ -512,97 +527,105 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             if (lane == 0) mbar_arrive(bar(kBarQFull + (k & 1)));
         }
     } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
-        // ------------------------- MMA issuers: warp 9 for warpgroup 0, warp 10 for warpgroup 1 -------------------------
-        // Slot number seq (counted over all items of the CTA) belongs to warpgroup seq % 2.  Each issuer
-        // walks every slot (observing each "landed" phase in order) and issues the MMAs of its own: S of
-        // own slot c goes into buffer c % 2 - free, because P V of own slot c - 2, which read P from
-        // it, was issued earlier by this same thread and the tensor pipe runs in order - and only then
-        // P V of own slot c - 1, once its P is there.
+        // ------------------------- Q K^T issuers: warp 9 for warpgroup 0, warp 10 for warpgroup 1 -------------------------
+        // Slot number seq (counted over all items of the CTA) belongs to warpgroup seq % 2 (the rings
+        // have an even number of slots, so a ring slot always serves the same warpgroup).  One thread
+        // issues MMAs too slowly to serve a warpgroup alone, so S and P V have an issuer each.  S of
+        // own slot c goes into buffer c % 2 as soon as K has landed and P V of own slot c - 2, which
+        // read P from that buffer, has completed: two slots ahead of the softmax.
         if (lane == 0) {
             constexpr uint32_t kIdescQK = instr_desc(kSlotTokens, 0);
-            constexpr uint32_t kIdescPV = instr_desc(HD, 1);
             const int wg = warp - kMmaWarp;
             const uint32_t qbase0 = sbase + kQOff;
             int seq = 0;                 // slots seen (all items, both warpgroups)
             int c = 0;                   // own slots issued
-            int pend_slot = -1, pend_seq = 0, pend_npg = 0, pend_c = 0, pend_item = 0;
-            bool pend_first = false;
             TCP_DECL;
             TCTRACE_DECL(wg);
-            auto flush_pv = [&]() {
-                if (pend_slot < 0) return;
-                TCTRACE(2048 + (pend_seq & 1023));
-                TCP_WAIT(1, wait_or_abort(bar(kBarPFull + wg * 2 + (pend_c & 1)), (uint32_t)(pend_c >> 1) & 1u));
-                TCTRACE(3072 + (pend_seq & 1023));
-                // the first P V of an item overwrites O: both warpgroups must have read out the previous item
-                if (pend_first && pend_item > 0) TCP_WAIT(2, wait_or_abort(bar(kBarEpiB), (uint32_t)(pend_item - 1) & 1u));
-                TCP_WAIT(5, wait_or_abort(bar(kBarFullV + pend_slot), (uint32_t)(pend_seq / kNV) & 1u));
-                TCTRACE(3072 + 512 + (pend_seq & 511));
-                if (!*s_abort) {
-                    tc_fence_after();
-                    const uint32_t vbase = sbase + kVOff + pend_slot * kKBytes;
-                    const uint32_t pcol = tmem + kColS + (uint32_t)(wg * 2 + (pend_c & 1)) * 64;
-                    TCP_WAIT(7, for (int j = 0; j < pend_npg; ++j) {
-                        const uint64_t bd = smem_desc(vbase + j * 2048, 8192, 1024);
-                        umma_ts(tmem + kColO + wg * 128, pcol + j * 8, bd, kIdescPV, (pend_first && j == 0) ? 0u : 1u);
-                    }
-                    tc_commit(bar(kBarODone + wg));
-                    tc_commit(bar(kBarEmptyV + pend_slot)));
-                }
-                pend_slot = -1;
-            };
             for (int k = 0; !*s_abort; ++k) {
                 const int e = k % kNI;
                 TCP_WAIT(3, wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u));
                 if (*s_abort) break;
                 const int item = s_item[e].item;
                 const int ngroups = s_item[e].num_groups;
-                const int num_pages = s_item[e].it.num_pages;
                 mbar_arrive(bar(kBarItemEmpty + e));
                 if (item < 0) break;
                 TCP_WAIT(4, wait_or_abort(bar(kBarQFull + (k & 1)), (uint32_t)(k >> 1) & 1u));
                 if (*s_abort) break;
-                bool first_own = true;
                 const uint32_t qbase = qbase0 + (k & 1) * kQBytes;
                 for (int g = 0; g < ngroups; ++g, ++seq) {
-                    if ((seq & 1) != wg) continue;   // ring sizes are even: a slot's every phase is this warpgroup's or never
+                    if ((seq & 1) != wg) continue;
                     const int slot = seq % kNK;
                     TCTRACE(1024 + (seq & 1023));
+                    if (c >= 2) TCP_WAIT(1, wait_or_abort(bar(kBarPVDone + wg * 2 + (c & 1)), (uint32_t)((c >> 1) - 1) & 1u));
                     TCP_WAIT(5, wait_or_abort(bar(kBarFullK + slot), (uint32_t)(seq / kNK) & 1u));
                     if (*s_abort) break;
                     TCTRACE(seq & 1023);
-#ifdef EXP_PVFIRST
-                    flush_pv();
-#endif
                     tc_fence_after();
                     const uint32_t kbase = sbase + slot * kKBytes;
                     const uint32_t scol = tmem + kColS + (uint32_t)(wg * 2 + (c & 1)) * 64;
+#ifdef EXP_HALFQK
+                    TCP_WAIT(6, for (int ks = 0; ks < HD / 32; ++ks) {
+#else
                     TCP_WAIT(6, for (int ks = 0; ks < HD / 16; ++ks) {
+#endif
                         const uint64_t ad = smem_desc(qbase + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
                         const uint64_t bd = smem_desc(kbase + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
                         umma_ss(scol, ad, bd, kIdescQK, ks > 0 ? 1u : 0u);
                     }
                     tc_commit(bar(kBarSFull + wg * 2 + (c & 1)));
                     tc_commit(bar(kBarEmptyK + slot)));   // K of the slot is free as soon as S is there
-                    flush_pv();   // P V of the previous own slot, after S of this one
-                    pend_slot = seq % kNV;
-                    pend_seq = seq;
-                    pend_npg = min(4, num_pages - g * 4);
-                    pend_c = c;
-                    pend_item = k;
-                    pend_first = first_own;
-                    first_own = false;
                     ++c;
                 }
                 if (*s_abort) break;
                 tc_commit(bar(kBarQEmpty + (k & 1)));   // this issuer's Q K^T of the item (if any) have completed
-                // the item's last P V goes out now rather than after the next item's first S: the
-                // warpgroups' epilogue waits for it
-                flush_pv();
             }
-            flush_pv();
             TCTRACE_END(wg);
             TCP_FLUSH(8 + 8 * wg);
+        }
+        __syncwarp();
+    } else if (warp == kPvWarp || warp == kPvWarp + 1) {
+        // ------------------------- P V issuers: warp 13 for warpgroup 0, warp 14 for warpgroup 1 -------------------------
+        if (lane == 0) {
+            constexpr uint32_t kIdescPV = instr_desc(HD, 1);
+            const int wg = warp - kPvWarp;
+            int seq = 0, c = 0;
+            for (int k = 0; !*s_abort; ++k) {
+                const int e = k % kNI;
+                wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u);
+                if (*s_abort) break;
+                const int item = s_item[e].item;
+                const int ngroups = s_item[e].num_groups;
+                const int num_pages = s_item[e].it.num_pages;
+                mbar_arrive(bar(kBarItemEmpty + e));
+                if (item < 0) break;
+                bool first_own = true;
+                for (int g = 0; g < ngroups; ++g, ++seq) {
+                    if ((seq & 1) != wg) continue;
+                    const int slot = seq % kNV;
+                    const int npg = min(4, num_pages - g * 4);
+                    wait_or_abort(bar(kBarPFull + wg * 2 + (c & 1)), (uint32_t)(c >> 1) & 1u);
+                    // the first P V of an item overwrites O: both warpgroups must have read out the previous item
+                    if (first_own && k > 0) wait_or_abort(bar(kBarEpiB), (uint32_t)(k - 1) & 1u);
+                    wait_or_abort(bar(kBarFullV + slot), (uint32_t)(seq / kNV) & 1u);
+                    if (*s_abort) break;
+                    tc_fence_after();
+                    const uint32_t vbase = sbase + kVOff + slot * kKBytes;
+                    const uint32_t pcol = tmem + kColS + (uint32_t)(wg * 2 + (c & 1)) * 64;
+#ifdef EXP_ONEPV
+                    for (int j = 0; j < 1; ++j) {
+#else
+                    for (int j = 0; j < npg; ++j) {
+#endif
+                        const uint64_t bd = smem_desc(vbase + j * 2048, 8192, 1024);
+                        umma_ts(tmem + kColO + wg * 128, pcol + j * 8, bd, kIdescPV, (first_own && j == 0) ? 0u : 1u);
+                    }
+                    tc_commit(bar(kBarPVDone + wg * 2 + (c & 1)));
+                    tc_commit(bar(kBarODone + wg));
+                    tc_commit(bar(kBarEmptyV + slot));
+                    first_own = false;
+                    ++c;
+                }
+            }
         }
         __syncwarp();
     }
@@ -625,8 +648,10 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 
         for (int k = 0; !*s_abort; ++k) {
             const int e = k % kNI;
+            TCTRACE(8);
             TCP_WAIT(1, wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u));
             if (*s_abort) break;
+            TCTRACE(9);
             const int item = s_item[e].item;
             const int ngroups = s_item[e].num_groups;
             const int it_num_tokens = s_item[e].it.num_tokens, it_num_pages = s_item[e].it.num_pages;
@@ -643,6 +668,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             const int64_t mb = s_rowbase[(k & 1) * 128 + row];
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarQEmpty + (k & 1)));   // row bases read
+            TCTRACE(10);
             float m = -INFINITY, l = 0.f;
             int citem = 0;      // own slots of this item
 
