@@ -618,6 +618,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #endif
                         const uint64_t bd = smem_desc(vbase + j * 2048, 8192, 1024);
                         umma_ts(tmem + kColO + wg * 128, pcol + j * 8, bd, kIdescPV, (first_own && j == 0) ? 0u : 1u);
+                        umma_ts(tmem + kColO + wg * 128, pcol + 32 + j * 8, bd, kIdescPV, 1u);   // the lower part of P
                     }
                     tc_commit(bar(kBarPVDone + wg * 2 + (c & 1)));
                     tc_commit(bar(kBarODone + wg));
@@ -746,33 +747,33 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     }
                 }
 
-                // p = 2^(s - m), its per-page sums, and the P row as bf16 pairs (A operand of P V)
+                // p = 2^(s - m), its per-page sums, and the P row as bf16 pairs (A operand of P V) in two
+                // parts: the upper 16 bits of p, and the rest rounded to bf16.  One bf16 alone carries
+                // 2^-9 relative error into the output, more than its tolerance when few tokens hold most of
+                // a row's mass; P V is accumulated over both parts.
                 float ps[4] = {0.f, 0.f, 0.f, 0.f};
-                uint32_t pk[32];
+                uint32_t pk[32], pl[32];
                 if (warp_has_rows) {
                     const float mm = valid ? m : 0.f;   // rows past the item's end: harmless, never read
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-#ifdef EXP_NOEXP
-                        const float p0 = (__uint_as_float(sr[(2 * j) >> 5][(2 * j) & 31]) - mm) * 0.001f;
-                        const float p1 = (__uint_as_float(sr[(2 * j + 1) >> 5][(2 * j + 1) & 31]) - mm) * 0.001f;
-#else
                         const float p0 = fast_exp2(__uint_as_float(sr[(2 * j) >> 5][(2 * j) & 31]) - mm);
                         const float p1 = fast_exp2(__uint_as_float(sr[(2 * j + 1) >> 5][(2 * j + 1) & 31]) - mm);
-#endif
                         ps[j >> 3] += p0;
                         ps[j >> 3] += p1;
-                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-                        pk[j] = *reinterpret_cast<const uint32_t*>(&b2);
+                        const uint32_t h0 = __float_as_uint(p0) & 0xffff0000u, h1 = __float_as_uint(p1) & 0xffff0000u;
+                        pk[j] = __byte_perm(h0, h1, 0x7632);   // (h1 upper half, h0 upper half)
+                        const __nv_bfloat162 lo2 = __floats2bfloat162_rn(p0 - __uint_as_float(h0), p1 - __uint_as_float(h1));
+                        pl[j] = *reinterpret_cast<const uint32_t*>(&lo2);
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) pk[j] = 0u;
+                    for (int j = 0; j < 32; ++j) pk[j] = pl[j] = 0u;
                 }
-                // over the first 32 columns of the S buffer, whose 64 values are all in registers by now
-#ifndef EXP_NOPST
+                // over the S buffer, whose 64 values are all in registers by now: upper parts in its
+                // first 32 columns, lower parts in the other 32
                 tmem_st32(scol, pk);
-#endif
+                tmem_st32(scol + 32, pl);
                 l += (ps[0] + ps[1]) + (ps[2] + ps[3]);
                 if (valid && a.block_mass != nullptr) {
 #pragma unroll

@@ -57,6 +57,16 @@ def test_row_counts_around_tile_edges(sharers, G):
     _parity(w)
 
 
+@pytest.mark.parametrize("ntok", [1, 3, 17, 64, 130])
+@pytest.mark.parametrize("q_gain", [1.0, 6.0])
+def test_short_shared_segment_on_the_tensor_core_path(ntok, q_gain):
+    # 16 sharers x G = 7 -> 112 stacked rows (the tcgen05 kernel) over a segment of a few tokens, alone:
+    # every probability is large, so the rounding of P to bf16 shows in the output if anywhere
+    w = workloads.make_from_segments("short_tc", 28, 4, 128, [ntok], [[0]] * 16, seed=40 + ntok, q_gain=q_gain)
+    err, plan = _parity(w)
+    assert any(plan.item(i)[8] == 1 for i in range(plan.num_work_items))
+
+
 def test_long_segment_many_chunks_and_custom_scale():
     w = workloads.make_from_segments("long", 8, 2, 128, [5000, 33, 700], [[0, 1], [0, 2], [0]], seed=13,
                                      sm_scale=0.11)
