@@ -135,6 +135,13 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     const int cap = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, fair * 2 / 3));
     const int base = (int)std::min<int64_t>(128, std::max<int64_t>(kMinChunk, fair / 6));
 
+    // Items of the tensor-core kernel are as long as three quarters of an SM's share of ALL the work:
+    // that kernel pays for every item (epilogue, hand-over) and once per CTA at its start, and the
+    // warp-MMA kernel, which starts on each SM as the tensor-core CTA there ends, takes up the slack
+    // of an uneven split.
+    const int tc_chunk = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, fair * 3 / 2));
+    int exp_tc_chunk = 0;   // development override
+    if (const char* e = std::getenv("RKSC_TC_CHUNK")) exp_tc_chunk = std::atoi(e);
     int64_t rows_total = 0;
     {
         size_t n_items = 0;   // exact count, so that the item vector is allocated once
@@ -145,7 +152,9 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
             const int nsb = ceil_div(ns, seg_rows_per_block(ns));
             for (int sb = 0; sb < nsb; ++sb) {
                 const int rows = ((int)((int64_t)ns * (sb + 1) / nsb) - (int)((int64_t)ns * sb / nsb)) * G;
-                n_items += (size_t)ceil_div(np, std::min(cap, std::max(base, 2 * rows))) * L.num_kv_heads;
+                int want0 = std::min(cap, std::max(base, 2 * rows));
+                if (tc_ok && rows >= kTcMinRows) want0 = exp_tc_chunk > 0 ? exp_tc_chunk : tc_chunk;
+                n_items += (size_t)ceil_div(np, want0) * L.num_kv_heads;
             }
         }
         P.items.reserve(n_items);
@@ -160,7 +169,8 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
             const int sh_lo = (int)((int64_t)ns * sb / nsb), sh_hi = (int)((int64_t)ns * (sb + 1) / nsb);
             const int rows = (sh_hi - sh_lo) * G;
             const int klass = (tc_ok && rows >= kTcMinRows) ? 1 : 0;
-            const int want = std::min(cap, std::max(base, 2 * rows));
+            int want = std::min(cap, std::max(base, 2 * rows));
+            if (klass == 1) want = exp_tc_chunk > 0 ? exp_tc_chunk : tc_chunk;
             const int nch = ceil_div(np, want);
             for (int c = 0; c < nch; ++c) {
                 const int p_lo = (int)((int64_t)np * c / nch), p_hi = (int)((int64_t)np * (c + 1) / nch);
