@@ -140,8 +140,6 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     // warp-MMA kernel, which starts on each SM as the tensor-core CTA there ends, takes up the slack
     // of an uneven split.
     const int tc_chunk = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, fair * 3 / 2));
-    int exp_tc_chunk = 0;   // development override
-    if (const char* e = std::getenv("RKSC_TC_CHUNK")) exp_tc_chunk = std::atoi(e);
     int64_t rows_total = 0;
     {
         size_t n_items = 0;   // exact count, so that the item vector is allocated once
@@ -153,7 +151,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
             for (int sb = 0; sb < nsb; ++sb) {
                 const int rows = ((int)((int64_t)ns * (sb + 1) / nsb) - (int)((int64_t)ns * sb / nsb)) * G;
                 int want0 = std::min(cap, std::max(base, 2 * rows));
-                if (tc_ok && rows >= kTcMinRows) want0 = exp_tc_chunk > 0 ? exp_tc_chunk : tc_chunk;
+                if (tc_ok && rows >= kTcMinRows) want0 = tc_chunk;
                 n_items += (size_t)ceil_div(np, want0) * L.num_kv_heads;
             }
         }
@@ -170,7 +168,7 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
             const int rows = (sh_hi - sh_lo) * G;
             const int klass = (tc_ok && rows >= kTcMinRows) ? 1 : 0;
             int want = std::min(cap, std::max(base, 2 * rows));
-            if (klass == 1) want = exp_tc_chunk > 0 ? exp_tc_chunk : tc_chunk;
+            if (klass == 1) want = tc_chunk;
             const int nch = ceil_div(np, want);
             for (int c = 0; c < nch; ++c) {
                 const int p_lo = (int)((int64_t)np * c / nch), p_hi = (int)((int64_t)np * (c + 1) / nch);
