@@ -349,9 +349,11 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
     if (warp == kProducerWarp) {
         // ------------------------------------ producer ------------------------------------
+        // CTA i starts with item i (no round trip to the counter before the first load); the counter
+        // hands out the items after the first gridDim.x
         auto claim = [&]() {
             int v = 0;
-            if (lane == 0) v = atomicAdd(a.counters + 2, 1);
+            if (lane == 0) v = (int)gridDim.x + atomicAdd(a.counters + 2, 1);
             return __shfl_sync(0xffffffffu, v, 0);
         };
         auto fetch_item = [&](int i) {
@@ -387,7 +389,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         // copies fast enough for the whole stream): K of a slot is needed two slots before its softmax
         // starts and is free again as soon as Q K^T has run, V is needed after the softmax.
         int seq = 0;
-        int idx = claim();
+        int idx = (int)blockIdx.x;
         WorkItem it = fetch_item(idx);
         publish(idx, it);
         int ids = fetch_ids(it, 0);
@@ -478,8 +480,21 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         // row goes to half c / 8, at chunk (c % 8) ^ (r % 8) of the row's 128 bytes (the 128-byte
         // swizzle the MMA's shared-memory descriptor expects).
         const int G = a.G;
+        // the CTA's first item is item blockIdx.x: fetched here, alongside the producer's own fetch,
+        // so that its sharers and query rows are on their way before the producer has published it
+        WorkItem it0{};
+        if ((int)blockIdx.x < a.num_tc_items) it0 = a.plan.items[blockIdx.x];
         for (int k = 0; !*s_abort; ++k) {
             const int e = k % kNI;
+            Sharer sh[4];
+            if (k == 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int r = lane + 32 * i;
+                    sh[i] = Sharer{};
+                    if (r < it0.num_sharers * G) sh[i] = a.plan.sharers[it0.sharer_begin + r / G];
+                }
+            }
             wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u);
             if (*s_abort) break;
             const int item = s_item[e].item;
@@ -489,12 +504,13 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             if (item < 0) break;
             const int rows = it.num_sharers * G;
             // the sharers of this lane's four rows, fetched before the wait below
-            Sharer sh[4];
+            if (k > 0) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int r = lane + 32 * i;
-                sh[i] = Sharer{};
-                if (r < rows) sh[i] = a.plan.sharers[it.sharer_begin + r / G];
+                for (int i = 0; i < 4; ++i) {
+                    const int r = lane + 32 * i;
+                    sh[i] = Sharer{};
+                    if (r < rows) sh[i] = a.plan.sharers[it.sharer_begin + r / G];
+                }
             }
             // this Q tile is free once every Q K^T of the item before the previous one has completed
             // and the softmax warps have read that item's row bases
