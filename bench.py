@@ -179,7 +179,8 @@ class DeviceBatch:
 
 
 def run_step(rk, batch: DeviceBatch, seg_events=None):
-    """One pass of the hot path.  Returns the plan (for byte counts).  3 kernel launches (2 without a gate)."""
+    """One pass of the hot path.  Returns the plan (for byte counts) and the number of kernel launches
+    (gate, tcgen05 segment kernel, warp segment kernel, merge; the plan knows which it needs)."""
     w = batch.w
     launches = 0
     if batch.has_gate:
@@ -200,7 +201,7 @@ def run_step(rk, batch: DeviceBatch, seg_events=None):
         rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=1, **kw)
         seg_events[1].record()
         rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=2, **kw)
-    launches += 2
+    launches += plan.num_kernel_launches
     return plan, launches
 
 
@@ -233,8 +234,10 @@ def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events, pool):
     w = batch.w
     g = w.gate
     n = len(ctxs)
+    launches = [0]
 
     def gate_stage(ctx):
+        launches[0] += 1
         rk.rksc_asks_gate(batch.h_branch, batch.h_root, batch.cand, g.alpha, g.tau,
                           branch_to_prefix=ctx.map_dev, sigma=ctx.sigma_dev, stream=ctx.stream)
         with torch.cuda.stream(ctx.stream):
@@ -255,6 +258,7 @@ def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events, pool):
             rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=1, **kw)
             ev[1].record(ctx.stream)
             rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=2, **kw)
+        launches[0] += plan.num_kernel_launches
         ctx.plan = plan                                # the context's previous plan is released here
 
     gate_stage(ctxs[0])
@@ -267,7 +271,7 @@ def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events, pool):
         nxt = pool.submit(plan_stage, ctxs[(i + 1) % n]) if i + 1 < steps else None
         attention_stage(ctxs[i % n], fut.result(), seg_events.get(i))
         fut = nxt
-    return 3 * steps
+    return launches[0]
 
 
 def attention_only_times(rk, batch: DeviceBatch, plan, iters: int, flush):

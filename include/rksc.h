@@ -149,6 +149,7 @@ typedef struct {
     int64_t duplicated_kv_tokens;/* sum over branches of the tokens they attend to        */
     int32_t on_device;           /* 1 when the lists were uploaded                        */
     int64_t num_pages_listed;    /* page ids in the tables (sum of the segments' pages)    */
+    int32_t num_kernel_launches; /* kernels one attention call launches with this plan     */
 } rksc_plan_info;
 
 RKSC_API int32_t rksc_plan_create(const rksc_layout* layout, const rksc_tables* tables, rksc_plan** out);

@@ -64,7 +64,8 @@ class _CPlanInfo(C.Structure):
     _fields_ = [("workspace_bytes", C.c_size_t), ("mass_elems", C.c_int64),
                 ("mass_off", C.POINTER(C.c_int64)), ("num_work_items", C.c_int32),
                 ("num_partial_rows", C.c_int32), ("unique_kv_tokens", C.c_int64),
-                ("duplicated_kv_tokens", C.c_int64), ("on_device", C.c_int32), ("num_pages_listed", C.c_int64)]
+                ("duplicated_kv_tokens", C.c_int64), ("on_device", C.c_int32), ("num_pages_listed", C.c_int64),
+                ("num_kernel_launches", C.c_int32)]
 
 
 def lib_path() -> str:
@@ -243,6 +244,7 @@ class Plan:
     duplicated_kv_tokens = property(lambda self: int(self._query().duplicated_kv_tokens))
     on_device = property(lambda self: bool(self._query().on_device))
     num_pages_listed = property(lambda self: int(self._query().num_pages_listed))
+    num_kernel_launches = property(lambda self: int(self._query().num_kernel_launches))
 
     @property
     def mass_off(self):

@@ -324,6 +324,8 @@ extern "C" RKSC_API int32_t rksc_plan_query(const rksc_plan* plan, rksc_plan_inf
     info->duplicated_kv_tokens = H.duplicated_kv_tokens;
     info->on_device = plan->on_device ? 1 : 0;
     info->num_pages_listed = (int64_t)H.seg_blocks.size();
+    info->num_kernel_launches = H.B == 0 ? 0 : (H.num_tc_items > 0 ? 1 : 0) +
+                                                   ((int)H.items.size() > H.num_tc_items ? 1 : 0) + 1;
     return RKSC_OK;
 }
 
