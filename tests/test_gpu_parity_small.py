@@ -67,6 +67,18 @@ def test_short_shared_segment_on_the_tensor_core_path(ntok, q_gain):
     assert any(plan.item(i)[8] == 1 for i in range(plan.num_work_items))
 
 
+@pytest.mark.parametrize("ntok", [16, 48, 100, 200])
+def test_many_short_items_per_cta_on_the_tensor_core_path(ntok):
+    # 300 segments x 4 KV heads = 1200 tensor-core items for 148 CTAs: every CTA runs through several
+    # items of one to four slots (its item ring wraps, items owned by one warpgroup only, epilogues
+    # with one accumulator empty), each shared by 3 branches x G = 7 -> 21 stacked rows
+    nseg = 300
+    w = workloads.make_from_segments("many_tc", 28, 4, 128, [ntok] * nseg,
+                                     [[s] for s in range(nseg) for _ in range(3)], seed=60 + ntok)
+    err, plan = _parity(w)
+    assert sum(1 for i in range(plan.num_work_items) if plan.item(i)[8] == 1) >= 1200
+
+
 def test_long_segment_many_chunks_and_custom_scale():
     w = workloads.make_from_segments("long", 8, 2, 128, [5000, 33, 700], [[0, 1], [0, 2], [0]], seed=13,
                                      sm_scale=0.11)
