@@ -8,26 +8,34 @@
 //   S[128 x 64]  = Q[128 x d] K^T        (tcgen05.mma, A = Q and B = K slot, both K-major in
 //                                         128-byte-swizzled shared memory)
 //   O[128 x d]  += P[128 x 64] V         (A = P read from tensor memory, B = V MN-major in smem)
-// with S, P and O in tensor memory.  One persistent CTA per SM, twelve warps:
+// with S, P and O in tensor memory.  One persistent CTA per SM, sixteen warps in four warpgroups:
 //   warps 0-3 / 4-7  two softmax warpgroups; thread = one stacked row (TMEM lane).  They take
 //                    alternate 64-token slots, each with two S buffers, its own O accumulator and
 //                    its own running (max, sum), merged at the end of the item.  Per slot: tcgen05.ld
 //                    of the S row, scale + mask + online softmax in base 2, per-page softmax mass
-//                    (log2, absolute) to global memory, P as bf16 written over the first half of the
-//                    same S buffer (tcgen05.st); O is rescaled in TMEM only when a running maximum
-//                    of the warp moved by more than 2^8.  A warpgroup's only wait per slot is "S ready".
-//   warp 8           producer: claims work items from a global counter, publishes their descriptors
-//                    in a small item ring and streams their pages by TMA (cp.async.bulk.tensor,
-//                    128-byte swizzle, no multicast) into a five-slot ring, four pages per slot.
-//   warps 9, 10      MMA issuers, one per warpgroup (one lane each; warp 9 also allocates TMEM): S of
-//                    the warpgroup's next slot is issued before P V of its previous one, into the S
-//                    buffer that P V before that has read, so S is waiting when the warpgroup comes
-//                    out of its softmax and the tensor pipe runs under both softmaxes.
-//   warp 11          Q loader: an item ahead, gathers the item's stacked query rows into the
-//                    swizzled Q tile (cp.async) and each row's block-mass base into shared memory.
-// Completion of MMAs is signalled with tcgen05.commit onto mbarriers (S ready, P V done / ring slot
-// free, Q tile free).  Every wait is bounded: on expiry the CTA records RKSC_ERR_DEVICE_TIMEOUT,
-// stops issuing work, skips further waits, frees its TMEM and returns.
+//                    (log2, absolute) to global memory, P written over the same S buffer in two bf16
+//                    parts (tcgen05.st); O is rescaled in TMEM only when a running maximum of the
+//                    warp moved by more than 2^8.  A warpgroup's only wait per slot is "S ready".
+//   warp 8           K producer: takes work items (the first by CTA index, then from a global counter),
+//                    publishes their descriptors in a small item ring and streams the K half of their
+//                    pages by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a
+//                    four-slot K ring, four pages per slot.
+//   warp 12          V producer: follows the item ring and streams the V halves into a four-slot V ring.
+//                    (One warp issues TMA copies at about 2.8 TB/s device-wide at most; and K, needed
+//                    two slots before a slot's softmax, and V, needed after it, would pin a common slot
+//                    four slot times.)
+//   warps 9, 10      Q K^T issuers, one per warpgroup (one lane each; warp 9 also allocates TMEM): S of
+//                    the warpgroup's slot c is issued once its K has landed and P V of slot c - 2 has
+//                    left the buffer, so S is waiting when the warpgroup comes out of its softmax.
+//   warps 13, 14     P V issuers, one per warpgroup.  (One thread issues a tcgen05.mma only every
+//                    100-150 cycles: a single issuer per warpgroup was busy the whole slot.)
+//   warp 11          Q loader: an item ahead, gathers the item's stacked query rows into one of two
+//                    swizzled Q tiles (cp.async) and each row's block-mass base into shared memory.
+//   warp 15          idle (it completes the fourth warpgroup, so that registers can be re-divided:
+//                    192 per softmax thread, 64 per helper thread).
+// Completion of MMAs is signalled with tcgen05.commit onto mbarriers (S ready, P V done / S buffer
+// free, ring slots free, Q tile free).  Every wait is bounded: on expiry the CTA records
+// RKSC_ERR_DEVICE_TIMEOUT, stops issuing work, skips further waits, frees its TMEM and returns.
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -46,13 +54,12 @@ constexpr int kPvWarp = kSmWarps + 5;             // 13 and 14: P V issuers of w
 constexpr int kTcThreads = (kSmWarps + 8) * 32;   // 512: four warpgroups (warp 15 idles), so that registers can be re-divided
 constexpr int kNK = 4;                            // K ring slots (even: a slot always serves the same warpgroup)
 constexpr int kNV = 4;                            // V ring slots (even)
-constexpr int kVLag = 4;                          // the V stream runs this many slots behind the K stream
 constexpr int kNI = 4;                            // item ring entries
 constexpr int kSlotTokens = 64;                   // 4 pages
 constexpr int kKBytes = kSlotTokens * HD * 2;     // K (or V) of a slot: [half][64 tokens][128 B] = 16 KiB
 constexpr int kVOff = kNK * kKBytes;
 constexpr int kRingBytes = (kNK + kNV) * kKBytes; // 128 KiB
-static_assert(kNK % 2 == 0 && kNV % 2 == 0 && kVLag >= 1 && kVLag < kNK + 4 && kVLag < 8, "ring geometry");
+static_assert(kNK % 2 == 0 && kNV % 2 == 0, "ring geometry");
 constexpr int kQOff = kRingBytes;                 // Q tiles [2 (item parity)][half][128 rows][128 B], 128-byte swizzle: 2 x 32 KiB
 constexpr int kQBytes = 128 * HD * 2;
 constexpr int kRowOff = kQOff + 2 * kQBytes;      // block-mass base of every row [2][128] int64
@@ -76,8 +83,7 @@ constexpr int kBarEpiA = kBarPVDone + 4;          //        item epilogue: (m, l
 constexpr int kBarEpiB = kBarEpiA + 1;            //        item epilogue: accumulators read
 constexpr int kNumBars = kBarEpiB + 1;
 constexpr int kItemOff = kBarOff + ((kNumBars * 8 + 15) / 16) * 16;
-constexpr int kVInfoOff = kItemOff + kNI * 64;    // [8] slots the K stream has issued and the V stream has not: 4 page ids, pages, KV head
-constexpr int kTmemPtrOff = kVInfoOff + 8 * 32;
+constexpr int kTmemPtrOff = kItemOff + kNI * 64;
 constexpr int kFlagOff = kTmemPtrOff + 16;
 constexpr int kSmemTotal = kFlagOff + 16;
 static_assert(kSmemTotal + 1024 <= 227 * 1024, "shared memory of the tcgen05 kernel");
@@ -242,11 +248,6 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-#ifdef EXP_STREAMONLY
-#define umma_ss(...)
-#define umma_ts(...)
-#define tc_commit(b) mbar_arrive(b)
-#endif
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -254,11 +255,6 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
 #ifdef RKSC_WAIT_PROFILE
 // Development aid: cycles one lane of each role spent in its waits.
 __device__ unsigned long long g_tc_prof[160][32];
-__device__ long long g_tc_trace[4][2048];
-__device__ int g_tc_trace_n[4];
-#define TCTRACE_DECL(w_) int tr_n = 0; const bool tr_on = blockIdx.x == 0 && (threadIdx.x & 31) == 0; long long* const tr_buf = g_tc_trace[w_]
-#define TCTRACE(ev) { if (tr_on && tr_n < 2048) { tr_buf[tr_n++] = (clock64() << 12) | (long long)((ev) & 4095); } }
-#define TCTRACE_END(w_) { if (tr_on) g_tc_trace_n[w_] = tr_n; }
 __device__ int g_tc_dbg[32][4];
 __device__ int g_tc_dbg_n, g_tc_dbg_n2;
 #define TCP_DECL unsigned long long tcp[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long tcp_begin = clock64()
@@ -268,9 +264,6 @@ __device__ int g_tc_dbg_n, g_tc_dbg_n2;
 #define TCP_DECL
 #define TCP_WAIT(i, stmt) stmt
 #define TCP_FLUSH(base)
-#define TCTRACE_DECL(w_)
-#define TCTRACE(ev)
-#define TCTRACE_END(w_)
 #endif
 
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -365,7 +358,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             return (first + lane < w.num_pages) ? __ldg(a.plan.seg_blocks + w.page_begin + first + lane) : 0;
         };
         TCP_DECL;
-        TCTRACE_DECL(2);
         int nitem = 0;   // item descriptors published
         auto publish = [&](int idx, const WorkItem& w) {
             const int e = nitem % kNI;
@@ -406,10 +398,8 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 // lane = 2 * page + half
                 const int page = __shfl_sync(0xffffffffu, ids, (g & 7) * 4 + ((lane >> 1) & 3));
                 if ((g & 7) == 7) ids = ids_ahead;
-                TCTRACE(1024 + (seq & 1023));
                 if (seq >= kNK) TCP_WAIT(1, wait_or_abort(bar(kBarEmptyK + kslot), (uint32_t)(seq / kNK - 1) & 1u));
                 if (*s_abort) break;
-                TCTRACE(seq & 1023);
                 const uint32_t full = bar(kBarFullK + kslot);
                 if (lane == 0) mbar_arrive_expect_tx(full, npg * (kBlock * HD * 2));
                 __syncwarp();
@@ -422,7 +412,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             it = nit;
             ids = fetch_ids(it, 0);
         }
-        TCTRACE_END(2);
         if (lane == 0) { TCP_FLUSH(0); }
         if (lane == 0) {   // the last CTA to stop claiming rewinds the counters for the next launch
             __threadfence();
@@ -556,7 +545,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             int seq = 0;                 // slots seen (all items, both warpgroups)
             int c = 0;                   // own slots issued
             TCP_DECL;
-            TCTRACE_DECL(wg);
             for (int k = 0; !*s_abort; ++k) {
                 const int e = k % kNI;
                 TCP_WAIT(3, wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u));
@@ -571,19 +559,13 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 for (int g = 0; g < ngroups; ++g, ++seq) {
                     if ((seq & 1) != wg) continue;
                     const int slot = seq % kNK;
-                    TCTRACE(1024 + (seq & 1023));
                     if (c >= 2) TCP_WAIT(1, wait_or_abort(bar(kBarPVDone + wg * 2 + (c & 1)), (uint32_t)((c >> 1) - 1) & 1u));
                     TCP_WAIT(5, wait_or_abort(bar(kBarFullK + slot), (uint32_t)(seq / kNK) & 1u));
                     if (*s_abort) break;
-                    TCTRACE(seq & 1023);
                     tc_fence_after();
                     const uint32_t kbase = sbase + slot * kKBytes;
                     const uint32_t scol = tmem + kColS + (uint32_t)(wg * 2 + (c & 1)) * 64;
-#ifdef EXP_HALFQK
-                    TCP_WAIT(6, for (int ks = 0; ks < HD / 32; ++ks) {
-#else
                     TCP_WAIT(6, for (int ks = 0; ks < HD / 16; ++ks) {
-#endif
                         const uint64_t ad = smem_desc(qbase + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
                         const uint64_t bd = smem_desc(kbase + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
                         umma_ss(scol, ad, bd, kIdescQK, ks > 0 ? 1u : 0u);
@@ -595,7 +577,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (*s_abort) break;
                 tc_commit(bar(kBarQEmpty + (k & 1)));   // this issuer's Q K^T of the item (if any) have completed
             }
-            TCTRACE_END(wg);
             TCP_FLUSH(8 + 8 * wg);
         }
         __syncwarp();
@@ -627,11 +608,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     tc_fence_after();
                     const uint32_t vbase = sbase + kVOff + slot * kKBytes;
                     const uint32_t pcol = tmem + kColS + (uint32_t)(wg * 2 + (c & 1)) * 64;
-#ifdef EXP_ONEPV
-                    for (int j = 0; j < 1; ++j) {
-#else
                     for (int j = 0; j < npg; ++j) {
-#endif
                         const uint64_t bd = smem_desc(vbase + j * 2048, 8192, 1024);
                         umma_ts(tmem + kColO + wg * 128, pcol + j * 8, bd, kIdescPV, (first_own && j == 0) ? 0u : 1u);
                         umma_ts(tmem + kColO + wg * 128, pcol + 32 + j * 8, bd, kIdescPV, 1u);   // the lower part of P
@@ -659,16 +636,11 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         int seq = 0;        // slots seen (all items, both warpgroups)
         int c = 0;          // own slots processed (all items)
         TCP_DECL;
-#ifdef RKSC_WAIT_PROFILE
-        int tr_n = 0; const bool tr_on = blockIdx.x == 0 && threadIdx.x == 0; long long* const tr_buf = g_tc_trace[3];
-#endif
 
         for (int k = 0; !*s_abort; ++k) {
             const int e = k % kNI;
-            TCTRACE(8);
             TCP_WAIT(1, wait_or_abort(bar(kBarItemFull + e), (uint32_t)(k / kNI) & 1u));
             if (*s_abort) break;
-            TCTRACE(9);
             const int item = s_item[e].item;
             const int ngroups = s_item[e].num_groups;
             const int it_num_tokens = s_item[e].it.num_tokens, it_num_pages = s_item[e].it.num_pages;
@@ -685,7 +657,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             const int64_t mb = s_rowbase[(k & 1) * 128 + row];
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarQEmpty + (k & 1)));   // row bases read
-            TCTRACE(10);
             float m = -INFINITY, l = 0.f;
             int citem = 0;      // own slots of this item
 
@@ -693,16 +664,10 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if ((seq & 1) != wg) continue;
                 // ---- this warpgroup's slot: S row -> softmax -> P row ----
                 const uint32_t scol = lane_addr + kColS + (uint32_t)(wg * 2 + (c & 1)) * 64;
-                TCTRACE(5);
                 TCP_WAIT(3, wait_or_abort(bar(kBarSFull + wg * 2 + (c & 1)), (uint32_t)(c >> 1) & 1u));
                 if (*s_abort) break;
                 tc_fence_after();
-                TCTRACE(6);
                 uint32_t sr[2][32];
-#ifdef EXP_STREAMONLY
-                for (int j = 0; j < 64; ++j) sr[j >> 5][j & 31] = 0u;
-                if (c >= 0) { __syncwarp(); if (lane == 0) mbar_arrive(bar(kBarPFull + wg * 2 + (c & 1))); ++c; ++citem; continue; }
-#endif
                 tmem_ld32(scol, sr[0]);
                 tmem_ld32(scol + 32, sr[1]);
                 tmem_wait_ld();
@@ -710,11 +675,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const int nvalid = it_num_tokens - g * kSlotTokens;   // tokens of this slot that exist
                 const int npg = min(4, it_num_pages - g * 4);
                 float mx = -INFINITY;
-#ifdef EXP_NOMAX
-                if (false) {
-#else
                 if (warp_has_rows) {
-#endif
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
                     if (nvalid >= kSlotTokens) {
 #pragma unroll
@@ -800,14 +761,12 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarPFull + wg * 2 + (c & 1)));
-                TCTRACE(7);
                 ++c;
                 ++citem;
             }
             if (*s_abort) break;
 
             // ---- item epilogue: merge the two warpgroups' states, write the partial ----
-            TCTRACE(1);
             const bool have_self = citem > 0;                 // warpgroup-uniform
             const bool have_oth = ngroups - citem > 0;        // the other warpgroup had a slot
             if (have_self) {
@@ -815,14 +774,12 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (*s_abort) break;
                 tc_fence_after();
             }
-            TCTRACE(2);
             s_ml[((k & 1) * 2 + wg) * 128 + row] = make_float2(m, l);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarEpiA));
             TCP_WAIT(5, wait_or_abort(bar(kBarEpiA), (uint32_t)k & 1u));
             if (*s_abort) break;
             tc_fence_after();
-            TCTRACE(3);
             {
                 const float2 oth = s_ml[((k & 1) * 2 + (1 - wg)) * 128 + row];
                 const float M = fmaxf(have_self ? m : -INFINITY, have_oth ? oth.x : -INFINITY);
@@ -845,11 +802,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         if (have_oth) v += c_oth * __uint_as_float(oo[j]);
                         os[j] = __float_as_uint(v);
                     }
-#ifdef EXP_NOEPIST
-                    if (valid && os[3] == 0x12345u) {
-#else
                     if (valid) {
-#endif
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
                             *reinterpret_cast<uint4*>(dst + q4 * 16 + j * 4) =
@@ -858,13 +811,11 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 }
                 if (valid && wg == 0) a.part_lse[(size_t)it_part_row_base + row] = M + fast_log2(L);
             }
-            TCTRACE(4);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarEpiB));   // the issuers wait for this before the next item's first P V
         }
 #ifdef RKSC_WAIT_PROFILE
-        if (tr_on) g_tc_trace_n[3] = tr_n;
         if (wg == 0 && quad == 0 && lane == 0) { tcp[6] = (unsigned long long)c; TCP_FLUSH(24); }
 #endif
     }
@@ -881,10 +832,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 }  // namespace
 
 #ifdef RKSC_WAIT_PROFILE
-extern "C" __attribute__((visibility("default"))) int rksc_debug_tc_trace(long long* host_out, int* n) {
-    if (cudaMemcpyFromSymbol(n, g_tc_trace_n, sizeof(g_tc_trace_n)) != cudaSuccess) return -1;
-    return cudaMemcpyFromSymbol(host_out, g_tc_trace, sizeof(g_tc_trace)) == cudaSuccess ? 0 : -1;
-}
 extern "C" __attribute__((visibility("default"))) int rksc_debug_tc_dbg(int* host_out) {
     return cudaMemcpyFromSymbol(host_out, g_tc_dbg, sizeof(g_tc_dbg)) == cudaSuccess ? 0 : -1;
 }
