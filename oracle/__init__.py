@@ -18,6 +18,10 @@ written for reading rather than speed:
                          softmax mass per KV block.
 * ``page_scores`` / ``rsbcm_evict`` - the eviction that consumes those masses
                          (Section 2.4, Algorithm 4).
+* ``suffix_prefill_attention`` / ``suffix_prefill_tables`` - the s suffix tokens of
+                         every branch attending causally on top of the shared cache
+                         (Appendix "Stepwise Batched Decode", step 1), and the tables
+                         that express it as a decode attention over B * s virtual branches.
 
 Parity pins: every function here is pinned by the CPU tests against closed
 forms, brute force on tiny inputs and invariants; none is "parity unpinned".
@@ -31,3 +35,4 @@ from .block_tables import (  # noqa: F401
 )
 from .branch_attention import branch_decode_attention, to_f32_numpy  # noqa: F401
 from .rsbcm import page_scores, rsbcm_evict, apply_eviction  # noqa: F401
+from .suffix_prefill import suffix_prefill_attention, suffix_prefill_tables  # noqa: F401
