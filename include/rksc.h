@@ -316,6 +316,33 @@ RKSC_API int32_t rksc_rsbcm_evict(const double* score, const int32_t* depth, int
  * ------------------------------------------------------------------------------------------ */
 RKSC_API int32_t rksc_tables_drop_evicted(const rksc_tables* in, const uint8_t* evicted, rksc_tables* out);
 
+/* ------------------------------------------------------------------------------------------
+ * Suffix prefill on the shared cache (paper Section 2.2, "KV broadcast and batched decode":
+ * y_b = f(s_b | C_B); Appendix "Stepwise Batched Decode", step (1)).  The s tokens of every
+ * branch's suffix are attended in one pass: query token i of branch b stands at position
+ * T_b - s + i of the branch's token sequence (the keys and values of the s tokens are the last s
+ * tokens the branch's tables list) and attends to every position up to and including its own.
+ *
+ * rksc_tables_for_suffix_prefill turns that into a decode attention over B * s virtual branches,
+ * which rksc_plan_create / rksc_branch_decode_attention then run on the same kernels: virtual
+ * branch b * s + i is query token i of branch b.  It lists every segment of b but the last
+ * unchanged (a shared prefix stays shared, now by s times as many rows), then two new segments
+ * cut from b's last segment: its pages that lie wholly before the first of the s tokens (shared
+ * by the s virtual branches of b; may be empty), and the pages from there up to the one holding
+ * token i, with only the tokens up to token i's own counted.  New segments are numbered after the S original ones:
+ * the common part of b is S + b * (s + 1), the part of token i is S + b * (s + 1) + 1 + i; a
+ * branch without segments gets s + 1 empty segments and s empty virtual branches.  The logical
+ * blocks of a virtual branch are the leading blocks of the branch in the same order (blocks that
+ * hold only later tokens are not listed), so block_mass of virtual branch b * s + i is the mass
+ * query token i puts on the branch's blocks.
+ * Call the attention with q [B * s][Hq][d] (token-major within a branch) and out likewise.
+ * Host arrays in, host arrays out; `out` is allocated by the library (rksc_tables_free).
+ * Errors: RKSC_ERR_INVALID_ARG (NULL, s < 1), RKSC_ERR_BAD_TABLE (inconsistent tables, or the
+ * last segment of a branch holds fewer than s tokens), RKSC_ERR_UNSUPPORTED (sizes beyond 2^30),
+ * RKSC_ERR_NOMEM.
+ * ------------------------------------------------------------------------------------------ */
+RKSC_API int32_t rksc_tables_for_suffix_prefill(const rksc_tables* in, int32_t s, rksc_tables* out);
+
 #ifdef __cplusplus
 }
 #endif

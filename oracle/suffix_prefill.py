@@ -23,7 +23,8 @@ def suffix_prefill_attention(num_q_heads, num_kv_heads, head_dim, sm_scale,
 
     q [B][s][Hq][d]; everything else as in branch_decode_attention.  Returns (out [B][s][Hq][d] fp64,
     list over branches of mass [s][Hq][nblk_b] fp64: the softmax mass query token i of head h puts on
-    the branch's j-th logical block).  A branch listing fewer than s tokens is an error.
+    the branch's j-th logical block).  A branch without tokens gets out = 0; one with some but
+    fewer than s tokens is an error.
     """
     q = np.asarray(q, dtype=np.float64)
     B, s = q.shape[0], q.shape[1]
@@ -35,10 +36,12 @@ def suffix_prefill_attention(num_q_heads, num_kv_heads, head_dim, sm_scale,
         Kd, Vd, blk, nblk_b = _gather_branch(b, seg_block_off, seg_blocks, seg_num_tokens,
                                              br_seg_off, br_segs, k_pool, v_pool)
         T = 0 if Kd is None else Kd.shape[1]
-        if T < s:
-            raise ValueError(f"branch {b} lists {T} tokens, fewer than the {s} suffix tokens")
         mass = np.zeros((s, num_q_heads, nblk_b), dtype=np.float64)
         masses[b] = mass
+        if T == 0:
+            continue                                  # a branch without tokens: out = 0, no masses
+        if T < s:
+            raise ValueError(f"branch {b} lists {T} tokens, fewer than the {s} suffix tokens")
         for i in range(s):
             Tv = T - s + i + 1                       # positions 0 .. T - s + i
             for h in range(num_q_heads):
@@ -57,11 +60,13 @@ def suffix_prefill_tables(seg_block_off, seg_blocks, seg_num_tokens, br_seg_off,
     Virtual branch b * s + i is query token i of branch b.  It lists every segment of b but the
     last unchanged, then two new segments cut from b's last segment: its pages that lie wholly
     before the first of the s tokens (shared by the s virtual branches of b, possibly empty), and
-    the pages from there to the end with only the tokens up to query token i's own counted.  New
+    the pages from there up to the one holding query token i, with only the tokens up to token i's
+    own counted.  New
     segments are numbered after the original ones, branch by branch: the common part of b is
     segment S + b * (s + 1), the part of token i is S + b * (s + 1) + 1 + i.  The last segment of a
     branch must hold at least s tokens.  A branch without segments yields s empty virtual branches.
-    The logical blocks of a virtual branch are those of the branch, in the same order.
+    The logical blocks of a virtual branch are the leading blocks of the branch, in the same order
+    (blocks that hold only later tokens are not listed).
     Returns a dict of int32 arrays with the five table fields.
     """
     S = len(seg_num_tokens)
@@ -88,9 +93,11 @@ def suffix_prefill_tables(seg_block_off, seg_blocks, seg_num_tokens, br_seg_off,
         off.append(len(blocks))
         ntok.append(ncommon * BLOCK)
         for i in range(s):
-            blocks.extend(int(x) for x in seg_blocks[lo + ncommon:hi])
+            nt = T - s + i + 1 - ncommon * BLOCK      # tokens of the tail part that token i sees (>= 1)
+            npg = (nt + BLOCK - 1) // BLOCK
+            blocks.extend(int(x) for x in seg_blocks[lo + ncommon:lo + ncommon + npg])
             off.append(len(blocks))
-            ntok.append(T - s + i + 1 - ncommon * BLOCK)
+            ntok.append(nt)
         for i in range(s):
             new_br_segs.extend(segs[:-1] + [S + b * (s + 1), S + b * (s + 1) + 1 + i])
             new_br_off.append(len(new_br_segs))

@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     rksc_rsbcm_workspace_bytes,
     rksc_rsbcm_evict,
     rksc_tables_drop_evicted,
+    rksc_tables_for_suffix_prefill,
     STATIC_WORKSPACE_BYTES,
     split_block_mass,
     EXPORTED_SYMBOLS,

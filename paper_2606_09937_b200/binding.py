@@ -35,6 +35,7 @@ EXPORTED_SYMBOLS = (
     "rksc_rsbcm_workspace_bytes",
     "rksc_rsbcm_evict",
     "rksc_tables_drop_evicted",
+    "rksc_tables_for_suffix_prefill",
 )
 STATIC_WORKSPACE_BYTES = 16 << 20
 
@@ -121,6 +122,8 @@ def lib() -> C.CDLL:
     L.rksc_rsbcm_evict.restype = C.c_int32
     L.rksc_rsbcm_evict.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_size_t, C.c_void_p]
+    L.rksc_tables_for_suffix_prefill.restype = C.c_int32
+    L.rksc_tables_for_suffix_prefill.argtypes = [C.POINTER(_CTables), C.c_int32, C.POINTER(_CTables)]
     L.rksc_tables_drop_evicted.restype = C.c_int32
     L.rksc_tables_drop_evicted.argtypes = [C.POINTER(_CTables), C.c_void_p, C.POINTER(_CTables)]
     _lib = L
@@ -425,6 +428,25 @@ def rksc_tables_drop_evicted(tables, evicted) -> Tables:
     out = _CTables()
     st = lib().rksc_tables_drop_evicted(C.byref(t.c), ev.ctypes.data_as(C.c_void_p), C.byref(out))
     _check(st, "rksc_tables_drop_evicted")
+    try:
+        S, B = out.num_segments, out.num_branches
+        cp = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(max(n, 1),))[:n].copy()
+        seg_block_off = cp(out.seg_block_off, S + 1)
+        br_seg_off = cp(out.br_seg_off, B + 1)
+        res = Tables(seg_block_off, cp(out.seg_blocks, int(seg_block_off[-1])), cp(out.seg_num_tokens, S),
+                     br_seg_off, cp(out.br_segs, int(br_seg_off[-1])))
+    finally:
+        lib().rksc_tables_free(C.byref(out))
+    return res
+
+
+def rksc_tables_for_suffix_prefill(tables, s: int) -> Tables:
+    """Host call: tables of the B * s virtual branches whose decode attention is the suffix prefill of
+    the last s tokens of every branch (see rksc_tables_for_suffix_prefill in rksc.h)."""
+    t = Tables.of(tables)
+    out = _CTables()
+    st = lib().rksc_tables_for_suffix_prefill(C.byref(t.c), int(s), C.byref(out))
+    _check(st, "rksc_tables_for_suffix_prefill")
     try:
         S, B = out.num_segments, out.num_branches
         cp = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(max(n, 1),))[:n].copy()

@@ -404,3 +404,99 @@ extern "C" RKSC_API int32_t rksc_tables_drop_evicted(const rksc_tables* in, cons
     out->br_segs = a4;
     return RKSC_OK;
 }
+
+// Tables that express the suffix prefill (Appendix "Stepwise Batched Decode", step 1) as a decode
+// attention over B * s virtual branches; the numbering is fixed by the header.
+extern "C" RKSC_API int32_t rksc_tables_for_suffix_prefill(const rksc_tables* in, int32_t s, rksc_tables* out) {
+    if (!in || !out || s < 1) return RKSC_ERR_INVALID_ARG;
+    std::memset(out, 0, sizeof(*out));
+    const int B = in->num_branches, S = in->num_segments;
+    if (B < 0 || S < 0 || !in->seg_block_off || !in->br_seg_off) return RKSC_ERR_INVALID_ARG;
+    if (S > 0 && !in->seg_num_tokens) return RKSC_ERR_INVALID_ARG;
+    if ((int64_t)B * s >= ((int64_t)1 << 30) || (int64_t)S + (int64_t)B * (s + 1) >= ((int64_t)1 << 30))
+        return RKSC_ERR_UNSUPPORTED;
+    if (in->seg_block_off[0] != 0 || in->br_seg_off[0] != 0) return RKSC_ERR_BAD_TABLE;
+    for (int sg = 0; sg < S; ++sg) {
+        const int64_t n = (int64_t)in->seg_block_off[sg + 1] - in->seg_block_off[sg];
+        const int64_t nt = in->seg_num_tokens[sg];
+        if (n < 0 || nt < 0 || nt > n * rksc::kBlock || (n > 0 && nt <= (n - 1) * rksc::kBlock)) return RKSC_ERR_BAD_TABLE;
+    }
+    const int64_t N = in->seg_block_off[S], R = in->br_seg_off[B];
+    if ((N > 0 && !in->seg_blocks) || (R > 0 && !in->br_segs)) return RKSC_ERR_INVALID_ARG;
+    // sizes
+    int64_t new_pages = N, new_refs = 0;
+    for (int b = 0; b < B; ++b) {
+        const int lo = in->br_seg_off[b], hi = in->br_seg_off[b + 1];
+        if (hi < lo) return RKSC_ERR_BAD_TABLE;
+        if (hi == lo) continue;
+        for (int i = lo; i < hi; ++i)
+            if (in->br_segs[i] < 0 || in->br_segs[i] >= S) return RKSC_ERR_BAD_TABLE;
+        const int last = in->br_segs[hi - 1];
+        const int64_t np = (int64_t)in->seg_block_off[last + 1] - in->seg_block_off[last];
+        const int64_t T = in->seg_num_tokens[last];
+        if (T < s) return RKSC_ERR_BAD_TABLE;
+        const int64_t ncommon = (T - s) / rksc::kBlock;
+        (void)np;
+        for (int i = 0; i < s; ++i) new_pages += (T - s + i + 1 - ncommon * rksc::kBlock + rksc::kBlock - 1) / rksc::kBlock;
+        new_pages += ncommon;
+        new_refs += (int64_t)s * ((hi - lo) + 1);
+    }
+    if (new_pages >= ((int64_t)1 << 31) || new_refs >= ((int64_t)1 << 31)) return RKSC_ERR_UNSUPPORTED;
+    const int S2 = S + B * (s + 1), B2 = B * s;
+    auto alloc = [](size_t n) { return (int32_t*)std::malloc(std::max<size_t>(1, n) * sizeof(int32_t)); };
+    int32_t* a0 = alloc((size_t)S2 + 1);
+    int32_t* a1 = alloc((size_t)new_pages);
+    int32_t* a2 = alloc((size_t)S2);
+    int32_t* a3 = alloc((size_t)B2 + 1);
+    int32_t* a4 = alloc((size_t)new_refs);
+    if (!a0 || !a1 || !a2 || !a3 || !a4) {
+        std::free(a0); std::free(a1); std::free(a2); std::free(a3); std::free(a4);
+        return RKSC_ERR_NOMEM;
+    }
+    std::memcpy(a0, in->seg_block_off, ((size_t)S + 1) * sizeof(int32_t));
+    if (N > 0) std::memcpy(a1, in->seg_blocks, (size_t)N * sizeof(int32_t));
+    if (S > 0) std::memcpy(a2, in->seg_num_tokens, (size_t)S * sizeof(int32_t));
+    int32_t pages = (int32_t)N, refs = 0;
+    a3[0] = 0;
+    for (int b = 0; b < B; ++b) {
+        const int lo = in->br_seg_off[b], hi = in->br_seg_off[b + 1];
+        const int seg0 = S + b * (s + 1);
+        if (hi == lo) {
+            for (int i = 0; i <= s; ++i) {
+                a0[seg0 + i + 1] = pages;
+                a2[seg0 + i] = 0;
+            }
+            for (int i = 0; i < s; ++i) a3[b * s + i + 1] = refs;
+            continue;
+        }
+        const int last = in->br_segs[hi - 1];
+        const int plo = in->seg_block_off[last], phi = in->seg_block_off[last + 1];
+        const int T = in->seg_num_tokens[last];
+        const int ncommon = (T - s) / rksc::kBlock;
+        for (int p = 0; p < ncommon; ++p) a1[pages++] = in->seg_blocks[plo + p];
+        a0[seg0 + 1] = pages;
+        a2[seg0] = ncommon * rksc::kBlock;
+        (void)phi;
+        for (int i = 0; i < s; ++i) {
+            const int nt = T - s + i + 1 - ncommon * rksc::kBlock;   // tokens of the tail part that token i sees
+            const int npg = (nt + rksc::kBlock - 1) / rksc::kBlock;
+            for (int p = 0; p < npg; ++p) a1[pages++] = in->seg_blocks[plo + ncommon + p];
+            a0[seg0 + 1 + i + 1] = pages;
+            a2[seg0 + 1 + i] = nt;
+        }
+        for (int i = 0; i < s; ++i) {
+            for (int j = lo; j < hi - 1; ++j) a4[refs++] = in->br_segs[j];
+            a4[refs++] = seg0;
+            a4[refs++] = seg0 + 1 + i;
+            a3[b * s + i + 1] = refs;
+        }
+    }
+    out->num_branches = B2;
+    out->num_segments = S2;
+    out->seg_block_off = a0;
+    out->seg_blocks = a1;
+    out->seg_num_tokens = a2;
+    out->br_seg_off = a3;
+    out->br_segs = a4;
+    return RKSC_OK;
+}
