@@ -516,6 +516,7 @@ def run_ours(args):
             line["e2e"] = run_e2e(rk, batch, kv_bytes, args.e2e_steps)
         if not args.no_sweep:
             line["configs"] = sweep_configs(rk, dev, flush, peak_gbs, skip=args.workload, cached=(args.workload, line))
+            line["suffix_prefill"] = suffix_prefill_measurement(rk, dev, flush, args.workload, 16)
         if not args.no_cpu_baseline:
             # about 10-30 s of oracle work: whole passes over the batch until 10 s have gone by
             passes, total, ub, cores, nb, Bt = 0, 0.0, 0, 1, 0, 0
@@ -646,6 +647,56 @@ def punch_long_context(rk, batch: DeviceBatch):
     batch.w = dataclasses.replace(w, tables=t, flat=None)
     batch.tables = holed
     return info
+
+
+def suffix_prefill_measurement(rk, dev, flush, workload: str, s: int):
+    """Suffix prefill (Appendix "Stepwise Batched Decode", step 1) on a config's tables: the last s tokens of
+    every branch's suffix attend causally on top of the shared cache, run as a decode attention over B * s
+    virtual branches (rksc_tables_for_suffix_prefill).  Attention call alone, cold L2."""
+    import torch
+    w = load_workload(workload)
+    b = DeviceBatch(w, dev)
+    plan0, _ = run_step(rk, b)                     # the decode step's plan: the tables the gate gave
+    torch.cuda.synchronize()
+    if b.has_gate:
+        f = w.flat
+        t = rk.rksc_tables_from_gate(b.map_host.numpy(), f.num_prefixes, f.shared_off, f.shared_pages, f.shared_ntok,
+                                     f.priv_off, f.priv_pages, f.priv_ntok, f.sfx_off, f.sfx_pages, f.sfx_ntok)
+    else:
+        t = b.tables
+    vt = rk.rksc_tables_for_suffix_prefill(t, s)
+    plan = rk.rksc_plan_create(b.layout, vt)
+    B, Hq, d = b.q.shape
+    g = torch.Generator(device="cpu").manual_seed(1234)
+    q = torch.randn((B * s, Hq, d), generator=g, dtype=torch.float32).to(torch.bfloat16).to(dev)
+    out = torch.empty((B * s, Hq, d), dtype=torch.float32, device=dev)
+    mass = torch.empty(max(plan.mass_elems, 1), dtype=torch.float32, device=dev)
+    ws = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device=dev)
+    kw = dict(out=out, block_mass=mass, workspace=ws, device_status=b.status)
+    times = []
+    for _ in range(12):
+        flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        rk.rksc_branch_decode_attention(plan, q, b.k_pool, b.v_pool, **kw)
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert int(b.status.item()) == 0
+    med = statistics.median(times[2:])
+    kv0, _ = algorithmic_bytes(plan0, b.w.layout)
+    lay = b.w.layout
+    flops = 4.0 * lay.head_dim * lay.num_q_heads * s * sum(
+        int(t.seg_num_tokens[sg]) for bb in range(B) for sg in t.br_segs[t.br_seg_off[bb]:t.br_seg_off[bb + 1]])
+    res = {"what": f"suffix prefill of s = {s} tokens per branch on {workload}: {B * s} virtual branches, "
+                   "attention call alone (segment kernels + merge), plan prebuilt, cold L2",
+           "ms_median": med, "query_tokens_per_s": B * s / (med * 1e-3),
+           "unique_kv_bytes_of_the_decode_tables": kv0, "tbps_on_those_bytes": kv0 / (med * 1e-3) / 1e12,
+           "kv_bytes_the_plan_reads": plan.unique_kv_tokens * 2 * lay.num_kv_heads * lay.head_dim * 2,
+           "attention_tflops": flops / (med * 1e-3) / 1e12, "work_items": plan.num_work_items}
+    del b
+    torch.cuda.empty_cache()
+    return res
 
 
 def sweep_configs(rk, dev, flush, peak_gbs, skip, cached):
