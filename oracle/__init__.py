@@ -23,6 +23,9 @@ written for reading rather than speed:
                          (Appendix "Stepwise Batched Decode", step 1), and the tables
                          that express it as a decode attention over B * s virtual branches.
 
+* ``logit_entropy`` / ``entropy_exit`` / ``generation_confidence`` / ``verify_skip`` - the
+                         numerics of CGEE (Section 2.3, Eq. 3-5, Algorithm 3).
+
 Parity pins: every function here is pinned by the CPU tests against closed
 forms, brute force on tiny inputs and invariants; none is "parity unpinned".
 """
@@ -36,3 +39,4 @@ from .block_tables import (  # noqa: F401
 from .branch_attention import branch_decode_attention, to_f32_numpy  # noqa: F401
 from .rsbcm import page_scores, rsbcm_evict, apply_eviction  # noqa: F401
 from .suffix_prefill import suffix_prefill_attention, suffix_prefill_tables  # noqa: F401
+from .cgee import logit_entropy, entropy_exit, generation_confidence, verify_skip  # noqa: F401
