@@ -343,6 +343,41 @@ RKSC_API int32_t rksc_tables_drop_evicted(const rksc_tables* in, const uint8_t* 
  * ------------------------------------------------------------------------------------------ */
 RKSC_API int32_t rksc_tables_for_suffix_prefill(const rksc_tables* in, int32_t s, rksc_tables* out);
 
+/* ------------------------------------------------------------------------------------------
+ * CGEE numerics (paper Section 2.3, "CGEE: Confidence-Gated Early Exit"; Algorithm 3).
+ *
+ * rksc_cgee_logit_entropy: for every row h_b of h (bf16 [B][D], device) the entropy, in nats, of
+ * p = softmax(h_b W_u^T) (Eq. 5) and its largest probability max_v p_v (the summand of the
+ * generation confidence, Eq. 3), fused with the unembedding product: W_u (bf16 [V][D], device,
+ * row-major) is read once per block of 16 rows of h and no logit is stored.  Products are bf16 x
+ * bf16 accumulated in fp32 on the tensor cores; the softmax statistics are fp32.
+ * entropy, top1_prob: device fp32 [B], either may be NULL (not both).  workspace: device, at least
+ * rksc_cgee_workspace_bytes() bytes, 16-byte aligned.  device_status (may be NULL): a device
+ * int32 that receives RKSC_ERR_DEVICE_TIMEOUT if a bounded wait inside the kernel ran out (the
+ * caller zeroes it).  Requires D a multiple of 8, D <= 4096 (the 16 rows of h stay in shared
+ * memory), h and w_u 16-byte aligned.
+ * Errors: RKSC_ERR_INVALID_ARG, RKSC_ERR_UNSUPPORTED (D, V >= 2^31), RKSC_ERR_WORKSPACE,
+ * RKSC_ERR_CUDA.
+ *
+ * rksc_cgee_entropy_exit: Algorithm 3's test for layer `layer`, per row:
+ * exit_flags[b] = (layer >= l_min && entropy[b] < theta && |entropy[b] - entropy_prev[b]| < eps),
+ * in fp32; entropy_prev = +inf before the first layer.  Device arrays [B].
+ *
+ * rksc_cgee_verify_skip: the Level-1 gate (Eq. 3 and 4).  top1_per_step is device fp32 [t][B]
+ * (the largest softmax probability of every decode step of every branch); confidence[b] (device
+ * [B], may be NULL) receives the mean over the t steps (summed in step order, fp32), and skip[0]
+ * (device int32) = (max_b p >= tau_conf && (max_b p - second largest) / max_b p >= r_gap), the
+ * second largest taken as 0 when B = 1; 0 when B = 0.
+ * ------------------------------------------------------------------------------------------ */
+RKSC_API size_t rksc_cgee_workspace_bytes(void);
+RKSC_API int32_t rksc_cgee_logit_entropy(const void* h, const void* w_u, int32_t B, int32_t D, int64_t V,
+                                         float* entropy, float* top1_prob, void* workspace,
+                                         size_t workspace_bytes, int32_t* device_status, void* stream);
+RKSC_API int32_t rksc_cgee_entropy_exit(const float* entropy, const float* entropy_prev, int32_t B, int32_t layer,
+                                        int32_t l_min, float theta, float eps, int32_t* exit_flags, void* stream);
+RKSC_API int32_t rksc_cgee_verify_skip(const float* top1_per_step, int32_t t, int32_t B, float tau_conf,
+                                       float r_gap, float* confidence, int32_t* skip, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,6 +27,9 @@ from .binding import (  # noqa: F401
     rksc_rsbcm_evict,
     rksc_tables_drop_evicted,
     rksc_tables_for_suffix_prefill,
+    rksc_cgee_logit_entropy,
+    rksc_cgee_entropy_exit,
+    rksc_cgee_verify_skip,
     STATIC_WORKSPACE_BYTES,
     split_block_mass,
     EXPORTED_SYMBOLS,

@@ -36,6 +36,10 @@ EXPORTED_SYMBOLS = (
     "rksc_rsbcm_evict",
     "rksc_tables_drop_evicted",
     "rksc_tables_for_suffix_prefill",
+    "rksc_cgee_workspace_bytes",
+    "rksc_cgee_logit_entropy",
+    "rksc_cgee_entropy_exit",
+    "rksc_cgee_verify_skip",
 )
 STATIC_WORKSPACE_BYTES = 16 << 20
 
@@ -122,6 +126,17 @@ def lib() -> C.CDLL:
     L.rksc_rsbcm_evict.restype = C.c_int32
     L.rksc_rsbcm_evict.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_size_t, C.c_void_p]
+    L.rksc_cgee_workspace_bytes.restype = C.c_size_t
+    L.rksc_cgee_workspace_bytes.argtypes = []
+    L.rksc_cgee_logit_entropy.restype = C.c_int32
+    L.rksc_cgee_logit_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    L.rksc_cgee_entropy_exit.restype = C.c_int32
+    L.rksc_cgee_entropy_exit.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_float,
+                                         C.c_void_p, C.c_void_p]
+    L.rksc_cgee_verify_skip.restype = C.c_int32
+    L.rksc_cgee_verify_skip.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_float, C.c_void_p, C.c_void_p,
+                                        C.c_void_p]
     L.rksc_tables_for_suffix_prefill.restype = C.c_int32
     L.rksc_tables_for_suffix_prefill.argtypes = [C.POINTER(_CTables), C.c_int32, C.POINTER(_CTables)]
     L.rksc_tables_drop_evicted.restype = C.c_int32
@@ -438,6 +453,54 @@ def rksc_tables_drop_evicted(tables, evicted) -> Tables:
     finally:
         lib().rksc_tables_free(C.byref(out))
     return res
+
+
+def rksc_cgee_logit_entropy(h, w_u, entropy=None, top1_prob=None, workspace=None, device_status=None, stream=None):
+    """Entropy (nats) and top-1 probability of softmax(h W_u^T) per row of h (Section 2.3, Eq. 5 / Eq. 3).
+    h bf16 [B][D], w_u bf16 [V][D] on the device.  Returns (entropy [B], top1_prob [B], device_status [1])."""
+    import torch
+    B, D = h.shape
+    V = w_u.shape[0]
+    dev = h.device
+    if entropy is None:
+        entropy = torch.empty(B, dtype=torch.float32, device=dev)
+    if top1_prob is None:
+        top1_prob = torch.empty(B, dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(int(lib().rksc_cgee_workspace_bytes()), dtype=torch.uint8, device=dev)
+    if device_status is None:
+        device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = lib().rksc_cgee_logit_entropy(h.data_ptr(), w_u.data_ptr(), B, D, V, entropy.data_ptr(), top1_prob.data_ptr(),
+                                       workspace.data_ptr(), workspace.numel(), device_status.data_ptr(),
+                                       _stream_ptr(stream, dev))
+    _check(st, "rksc_cgee_logit_entropy")
+    return entropy, top1_prob, device_status
+
+
+def rksc_cgee_entropy_exit(entropy, entropy_prev, layer: int, l_min: int, theta: float, eps: float, exit_flags=None,
+                           stream=None):
+    """Algorithm 3's exit test per row (device fp32 arrays [B]); returns int32 flags [B]."""
+    import torch
+    B = int(entropy.numel())
+    if exit_flags is None:
+        exit_flags = torch.empty(B, dtype=torch.int32, device=entropy.device)
+    st = lib().rksc_cgee_entropy_exit(entropy.data_ptr(), entropy_prev.data_ptr(), B, int(layer), int(l_min), float(theta),
+                                      float(eps), exit_flags.data_ptr(), _stream_ptr(stream, entropy.device))
+    _check(st, "rksc_cgee_entropy_exit")
+    return exit_flags
+
+
+def rksc_cgee_verify_skip(top1_per_step, tau_conf: float, r_gap: float, stream=None):
+    """Level-1 gate (Eq. 3, 4): top1_per_step device fp32 [t][B] -> (confidence [B], skip int32 [1])."""
+    import torch
+    t, B = top1_per_step.shape
+    dev = top1_per_step.device
+    conf = torch.empty(B, dtype=torch.float32, device=dev)
+    skip = torch.empty(1, dtype=torch.int32, device=dev)
+    st = lib().rksc_cgee_verify_skip(top1_per_step.data_ptr(), t, B, float(tau_conf), float(r_gap), conf.data_ptr(),
+                                     skip.data_ptr(), _stream_ptr(stream, dev))
+    _check(st, "rksc_cgee_verify_skip")
+    return conf, skip
 
 
 def rksc_tables_for_suffix_prefill(tables, s: int) -> Tables:

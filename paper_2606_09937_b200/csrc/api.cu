@@ -636,3 +636,108 @@ extern "C" RKSC_API int32_t rksc_rsbcm_evict(const double* score, const int32_t*
     }
     return RKSC_OK;
 }
+
+// ---- CGEE numerics (Section 2.3: Eq. 3-5, Algorithm 3) ----
+
+namespace {
+// A row-major bf16 matrix [rows][cols] fetched in boxes of box_rows x 64 columns, 128-byte swizzle.
+int32_t make_matrix_map(const void* base, int64_t rows, int cols, int box_rows, CUtensorMap* tm) {
+    EncodeTiledFn enc;
+    int32_t st = get_encode(&enc);
+    if (st != RKSC_OK) return st;
+    const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? RKSC_OK : RKSC_ERR_CUDA;
+}
+constexpr int kCgeeMaxParts = 1024;   // CTAs whose partial results the workspace holds
+}  // namespace
+
+extern "C" RKSC_API size_t rksc_cgee_workspace_bytes(void) { return (size_t)kCgeeMaxParts * 16 * 3 * sizeof(float); }
+
+extern "C" RKSC_API int32_t rksc_cgee_logit_entropy(const void* h, const void* w_u, int32_t B, int32_t D, int64_t V,
+                                                    float* entropy, float* top1_prob, void* workspace,
+                                                    size_t workspace_bytes, int32_t* device_status, void* stream) {
+    if (B < 0 || D <= 0 || V <= 0) return RKSC_ERR_INVALID_ARG;
+    if (B == 0) return RKSC_OK;
+    if (!h || !w_u || (!entropy && !top1_prob)) return RKSC_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(h) & 15) || (reinterpret_cast<uintptr_t>(w_u) & 15)) return RKSC_ERR_INVALID_ARG;
+    if (D % 8 != 0 || V >= ((int64_t)1 << 31)) return RKSC_ERR_UNSUPPORTED;   // TMA: row pitch a multiple of 16 bytes
+    if (!workspace || workspace_bytes < rksc_cgee_workspace_bytes() || (reinterpret_cast<uintptr_t>(workspace) & 15))
+        return RKSC_ERR_WORKSPACE;
+    int dev = -1;
+    int32_t st = ensure_device(&dev);
+    if (st != RKSC_OK) return st;
+    const size_t smem = cgee_smem_bytes(D);
+    if (smem > 227 * 1024 - 256) return RKSC_ERR_UNSUPPORTED;   // the hidden rows must fit in shared memory (D <= 4096)
+    static bool configured[kMaxDevices] = {};
+    static int sms[kMaxDevices] = {};
+    if (!configured[dev]) {
+        if (configure_cgee_kernel(227 * 1024 - 256) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            g_last_cuda = cudaGetLastError();
+            return RKSC_ERR_CUDA;
+        }
+        configured[dev] = true;
+    }
+    const int64_t ntiles = (V + 127) / 128;
+    const int grid = (int)std::min<int64_t>(std::min<int64_t>(ntiles, std::max(1, sms[dev])), kCgeeMaxParts);
+    CUtensorMap tm_w;
+    st = make_matrix_map(w_u, V, D, 128, &tm_w);
+    if (st != RKSC_OK) return st;
+    const int rows_per = cgee_rows_per_launch();
+    // more rows than one launch takes: row blocks one after another (W_u is read once per block)
+    for (int b0 = 0; b0 < B; b0 += rows_per) {
+        const int nb = std::min(rows_per, B - b0);
+        CUtensorMap tm_h;
+        st = make_matrix_map(static_cast<const uint8_t*>(h) + (size_t)b0 * D * 2, nb, D, rows_per, &tm_h);
+        if (st != RKSC_OK) return st;
+        cudaError_t e = launch_logit_entropy(tm_w, tm_h, nb, D, V, grid, static_cast<float*>(workspace),
+                                             entropy ? entropy + b0 : nullptr, top1_prob ? top1_prob + b0 : nullptr,
+                                             device_status, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) {
+            g_last_cuda = e;
+            cudaGetLastError();
+            return RKSC_ERR_CUDA;
+        }
+    }
+    return RKSC_OK;
+}
+
+extern "C" RKSC_API int32_t rksc_cgee_entropy_exit(const float* entropy, const float* entropy_prev, int32_t B, int32_t layer,
+                                                   int32_t l_min, float theta, float eps, int32_t* exit_flags,
+                                                   void* stream) {
+    if (B < 0) return RKSC_ERR_INVALID_ARG;
+    if (B == 0) return RKSC_OK;
+    if (!entropy || !entropy_prev || !exit_flags) return RKSC_ERR_INVALID_ARG;
+    int32_t st = ensure_device(nullptr);
+    if (st != RKSC_OK) return st;
+    cudaError_t e = launch_entropy_exit(entropy, entropy_prev, B, layer, l_min, theta, eps, exit_flags,
+                                        static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda = e;
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    return RKSC_OK;
+}
+
+extern "C" RKSC_API int32_t rksc_cgee_verify_skip(const float* top1_per_step, int32_t t, int32_t B, float tau_conf,
+                                                  float r_gap, float* confidence, int32_t* skip, void* stream) {
+    if (t < 1 || B < 0 || !skip) return RKSC_ERR_INVALID_ARG;
+    if (B > 0 && !top1_per_step) return RKSC_ERR_INVALID_ARG;
+    int32_t st = ensure_device(nullptr);
+    if (st != RKSC_OK) return st;
+    cudaError_t e = launch_verify_skip(top1_per_step, t, B, tau_conf, r_gap, confidence, skip,
+                                       static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda = e;
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    return RKSC_OK;
+}

@@ -47,6 +47,17 @@ cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream);
 cudaError_t launch_page_scores(const int2* chunks, int num_chunks, const int32_t* seg_block_off,
                                const int32_t* seg_sharer_off, const Sharer* sharers, const float* mass, double* score,
                                int Hq, cudaStream_t stream);
+// CGEE numerics (Section 2.3): entropy and top-1 probability of softmax(h W_u^T) for up to
+// cgee_rows_per_launch() rows of h; exit test; verify-skip gate.
+size_t cgee_smem_bytes(int D);
+int cgee_rows_per_launch();
+cudaError_t configure_cgee_kernel(int max_smem);
+cudaError_t launch_logit_entropy(const CUtensorMap& tm_w, const CUtensorMap& tm_h, int B, int D, long long V, int grid,
+                                 float* partial, float* entropy, float* top1, int32_t* status, cudaStream_t stream);
+cudaError_t launch_entropy_exit(const float* H, const float* H_prev, int B, int layer, int l_min, float theta, float eps,
+                                int32_t* flags, cudaStream_t stream);
+cudaError_t launch_verify_skip(const float* top1_steps, int t, int B, float tau_conf, float r_gap, float* p_out,
+                               int32_t* skip, cudaStream_t stream);
 cudaError_t launch_rsbcm_select(const double* score, const int32_t* depth, int32_t n, uint32_t k, uint64_t* keys,
                                 uint8_t* evicted, int32_t* num_evicted, cudaStream_t stream);
 

@@ -26,6 +26,7 @@ from .generators import (  # noqa: F401
     lowest_mass_pages,
     make_block_masses,
     make_eviction_inputs,
+    make_cgee_inputs,
     unique_kv_bytes,
     duplicated_kv_bytes,
     CONFIG_NAMES,

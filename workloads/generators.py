@@ -444,6 +444,20 @@ def make_eviction_inputs(n: int, seed: int = SEED_BASE + 51, max_depth: int = 6,
     return score, depth
 
 
+def make_cgee_inputs(B: int, D: int, V: int, seed: int = SEED_BASE + 60, logit_std: float = 3.0, peaked_rows=()):
+    """Synthetic inputs of the entropy hook: hidden rows h [B][D] and an unembedding matrix W_u [V][D],
+    both bf16 (torch), drawn so that the logits h W_u^T are about N(0, logit_std^2) - an entropy a few nats
+    below log V, as for a model some layers into its verify pass.  Rows in ``peaked_rows`` are aligned with
+    one vocabulary row each (a concentrated distribution: small entropy, top-1 probability near 1)."""
+    gen = _torch_gen(seed, 7)
+    w = torch.randn((V, D), generator=gen, dtype=torch.float32) / math.sqrt(D)
+    h = torch.randn((B, D), generator=gen, dtype=torch.float32) * logit_std
+    for i, b in enumerate(peaked_rows):
+        v = (977 * (i + 1)) % V
+        h[b] = w[v] * (12.0 / float(w[v].pow(2).sum()))      # that row's logit is 12, the others stay near 0
+    return h.to(torch.bfloat16), w.to(torch.bfloat16)
+
+
 def make_config(name: str, **kw) -> Workload:
     if name == "tiny":
         return make_tiny(**kw)
