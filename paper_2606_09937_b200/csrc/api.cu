@@ -672,7 +672,7 @@ extern "C" RKSC_API int32_t rksc_cgee_logit_entropy(const void* h, const void* w
     int dev = -1;
     int32_t st = ensure_device(&dev);
     if (st != RKSC_OK) return st;
-    const size_t smem = cgee_smem_bytes(D);
+    const size_t smem = cgee_smem_bytes(D, 16);
     if (smem > 227 * 1024 - 256) return RKSC_ERR_UNSUPPORTED;   // the hidden rows must fit in shared memory (D <= 4096)
     static bool configured[kMaxDevices] = {};
     static int sms[kMaxDevices] = {};
@@ -694,7 +694,7 @@ extern "C" RKSC_API int32_t rksc_cgee_logit_entropy(const void* h, const void* w
     for (int b0 = 0; b0 < B; b0 += rows_per) {
         const int nb = std::min(rows_per, B - b0);
         CUtensorMap tm_h;
-        st = make_matrix_map(static_cast<const uint8_t*>(h) + (size_t)b0 * D * 2, nb, D, rows_per, &tm_h);
+        st = make_matrix_map(static_cast<const uint8_t*>(h) + (size_t)b0 * D * 2, nb, D, nb <= 8 ? 8 : rows_per, &tm_h);
         if (st != RKSC_OK) return st;
         cudaError_t e = launch_logit_entropy(tm_w, tm_h, nb, D, V, grid, static_cast<float*>(workspace),
                                              entropy ? entropy + b0 : nullptr, top1_prob ? top1_prob + b0 : nullptr,

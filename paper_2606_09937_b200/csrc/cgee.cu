@@ -24,7 +24,9 @@ namespace {
 
 constexpr int kCgWarps = 8;                       // consumer warps
 constexpr int kCgThreads = (kCgWarps + 1) * 32;   // + producer
-constexpr int kCgStages = 6;
+// Stages of the W ring: six beside 16 hidden rows (112 KiB at D = 3584), ten beside 8 - the kernel
+// is bound by HBM latency x bytes in flight, and 96 KiB per SM in flight gives 4.9 TB/s.
+template <int NT> struct CgCfg { static constexpr int kStages = NT == 1 ? 10 : 6; };
 constexpr int kCgTileRows = 128;                  // vocabulary rows per tile
 constexpr int kCgStageBytes = kCgTileRows * 128;  // [128 rows][64 bf16]
 constexpr int kCgRows = 16;                       // hidden-state rows per launch
@@ -102,15 +104,18 @@ __device__ __forceinline__ Stat stat_merge(const Stat& a, const Stat& b) {
     return r;
 }
 
+template <int NT>
 __global__ void __launch_bounds__(kCgThreads, 1)
 logit_entropy_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, int D,
                      long long V, float* __restrict__ partial, int32_t* __restrict__ status) {
     extern __shared__ uint8_t cg_smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(cg_smem_raw) + 1023) & ~uintptr_t(1023));
+    constexpr int kCgStages = CgCfg<NT>::kStages;
+    constexpr int kHChunk = NT * 1024;                     // bytes of one 64-column chunk of the 8 * NT hidden rows
     const int nkc = (D + 63) / 64;                         // 64-column chunks of the hidden dimension
     const uint32_t ring = cg_smem_u32(smem);
-    const uint32_t hbase = ring + kCgStages * kCgStageBytes;   // [nkc][16 rows][128 B]
-    const uint32_t bars = hbase + nkc * 2048;              // full[stages], empty[stages], h
+    const uint32_t hbase = ring + kCgStages * kCgStageBytes;   // [nkc][8 * NT rows][128 B]
+    const uint32_t bars = hbase + nkc * kHChunk;           // full[stages], empty[stages], h
     // per-warp triples of the final merge: over the ring's first stage, which is idle by then
     float (*s_part)[kCgRows][3] = reinterpret_cast<float (*)[kCgRows][3]>(smem);
     __shared__ int s_abort;
@@ -138,8 +143,8 @@ logit_entropy_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
     if (warp == kCgWarps) {
         // ---------------- producer ----------------
         if (lane == 0) {
-            cg_mbar_expect_tx(bars + 8 * 2 * kCgStages, (uint32_t)nkc * 2048u);
-            for (int kc = 0; kc < nkc; ++kc) cg_tma_2d(hbase + kc * 2048, &tm_h, kc * 64, 0, bars + 8 * 2 * kCgStages);
+            cg_mbar_expect_tx(bars + 8 * 2 * kCgStages, (uint32_t)nkc * (uint32_t)kHChunk);
+            for (int kc = 0; kc < nkc; ++kc) cg_tma_2d(hbase + kc * kHChunk, &tm_h, kc * 64, 0, bars + 8 * 2 * kCgStages);
             uint32_t seq = 0;
             for (long long tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x) {
                 for (int kc = 0; kc < nkc && !*abort_flag; ++kc, ++seq) {
@@ -169,14 +174,29 @@ logit_entropy_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
                 wait_or_abort(bars + 8 * sg, (seq / kCgStages) & 1u);
                 if (*abort_flag) break;
                 const uint32_t wrow = ring + sg * kCgStageBytes + (16 * warp + a_row) * 128;
-                const uint32_t hrow = hbase + kc * 2048 + b_row * 128;
+                if (NT == 2) {
+                    const uint32_t hrow = hbase + kc * kHChunk + b_row * 128;
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    uint32_t a[4], b[4];
-                    cg_ldmatrix_x4(wrow + (((ks * 2 + a_chunk) ^ (a_row & 7)) << 4), a);
-                    cg_ldmatrix_x4(hrow + (((ks * 2 + b_chunk) ^ (b_row & 7)) << 4), b);
-                    cg_mma(c0, a, b[0], b[1]);
-                    cg_mma(c1, a, b[2], b[3]);
+                    for (int ks = 0; ks < 4; ++ks) {
+                        uint32_t a[4], b[4];
+                        cg_ldmatrix_x4(wrow + (((ks * 2 + a_chunk) ^ (a_row & 7)) << 4), a);
+                        cg_ldmatrix_x4(hrow + (((ks * 2 + b_chunk) ^ (b_row & 7)) << 4), b);
+                        cg_mma(c0, a, b[0], b[1]);
+                        cg_mma(c1, a, b[2], b[3]);
+                    }
+                } else {
+                    // 8 hidden rows: one ldmatrix.x4 brings the B fragments of two k-steps
+                    // (lanes 0-7: k-step 2j low half, 8-15: high half, 16-23 and 24-31: k-step 2j + 1)
+                    const uint32_t hrow = hbase + kc * kHChunk + (lane & 7) * 128;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        uint32_t b[4], a0[4], a1[4];
+                        cg_ldmatrix_x4(hrow + ((((j * 4) + (lane >> 3)) ^ (lane & 7)) << 4), b);
+                        cg_ldmatrix_x4(wrow + ((((2 * j) * 2 + a_chunk) ^ (a_row & 7)) << 4), a0);
+                        cg_ldmatrix_x4(wrow + ((((2 * j + 1) * 2 + a_chunk) ^ (a_row & 7)) << 4), a1);
+                        cg_mma(c0, a0, b[0], b[1]);
+                        cg_mma(c0, a1, b[2], b[3]);
+                    }
                 }
                 __syncwarp();
                 if (lane == 0) cg_mbar_arrive(bars + 8 * (kCgStages + sg));
@@ -187,14 +207,18 @@ logit_entropy_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
             if (v0 < V) {
                 stat_add(st[0], c0[0]);
                 stat_add(st[1], c0[1]);
-                stat_add(st[2], c1[0]);
-                stat_add(st[3], c1[1]);
+                if (NT == 2) {
+                    stat_add(st[2], c1[0]);
+                    stat_add(st[3], c1[1]);
+                }
             }
             if (v0 + 8 < V) {
                 stat_add(st[0], c0[2]);
                 stat_add(st[1], c0[3]);
-                stat_add(st[2], c1[2]);
-                stat_add(st[3], c1[3]);
+                if (NT == 2) {
+                    stat_add(st[2], c1[2]);
+                    stat_add(st[3], c1[3]);
+                }
             }
         }
         // the eight lanes with the same t hold disjoint vocabulary rows of the same hidden rows
@@ -295,16 +319,23 @@ __global__ void verify_skip_kernel(const float* __restrict__ top1_steps, int t, 
 
 }  // namespace
 
-size_t cgee_smem_bytes(int D) { return (size_t)kCgStages * kCgStageBytes + (size_t)((D + 63) / 64) * 2048 + (2 * kCgStages + 1) * 8 + 1024 + 64; }
+size_t cgee_smem_bytes(int D, int B) {
+    const int nt = B <= 8 ? 1 : 2;
+    const int stages = nt == 1 ? CgCfg<1>::kStages : CgCfg<2>::kStages;
+    return (size_t)stages * kCgStageBytes + (size_t)((D + 63) / 64) * nt * 1024 + (2 * stages + 1) * 8 + 1024 + 64;
+}
 int cgee_rows_per_launch() { return kCgRows; }
 
 cudaError_t configure_cgee_kernel(int max_smem) {
-    return cudaFuncSetAttribute(logit_entropy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    cudaError_t e = cudaFuncSetAttribute(logit_entropy_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(logit_entropy_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
 }
 
 cudaError_t launch_logit_entropy(const CUtensorMap& tm_w, const CUtensorMap& tm_h, int B, int D, long long V, int grid,
                                  float* partial, float* entropy, float* top1, int32_t* status, cudaStream_t stream) {
-    logit_entropy_kernel<<<grid, kCgThreads, cgee_smem_bytes(D), stream>>>(tm_w, tm_h, D, V, partial, status);
+    if (B <= 8) logit_entropy_kernel<1><<<grid, kCgThreads, cgee_smem_bytes(D, B), stream>>>(tm_w, tm_h, D, V, partial, status);
+    else logit_entropy_kernel<2><<<grid, kCgThreads, cgee_smem_bytes(D, B), stream>>>(tm_w, tm_h, D, V, partial, status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     logit_entropy_finish_kernel<<<1, kCgRows, 0, stream>>>(partial, grid, B, entropy, top1);

@@ -49,7 +49,7 @@ cudaError_t launch_page_scores(const int2* chunks, int num_chunks, const int32_t
                                int Hq, cudaStream_t stream);
 // CGEE numerics (Section 2.3): entropy and top-1 probability of softmax(h W_u^T) for up to
 // cgee_rows_per_launch() rows of h; exit test; verify-skip gate.
-size_t cgee_smem_bytes(int D);
+size_t cgee_smem_bytes(int D, int B);
 int cgee_rows_per_launch();
 cudaError_t configure_cgee_kernel(int max_smem);
 cudaError_t launch_logit_entropy(const CUtensorMap& tm_w, const CUtensorMap& tm_h, int B, int D, long long V, int grid,
