@@ -61,6 +61,8 @@ def parse_args():
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-config attention-only table")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-pipeline", action="store_true", help="time the steps strictly one after another")
+    ap.add_argument("--cgee-only", action="store_true",
+                    help="run only the CGEE entropy-kernel measurement and print its object (used for profiling)")
     return ap.parse_args()
 
 
@@ -390,15 +392,21 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    w = load_workload(args.workload, seed_shift=rank)
-    batch = DeviceBatch(w, dev)
-    if w.name == "long_context":
-        punch_long_context(rk, batch)
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
     flush_buf = torch.empty(max(2 * l2_bytes, 256 << 20), dtype=torch.uint8, device=dev)
 
     def flush():
         flush_buf.fill_(1)
+
+    if args.cgee_only:
+        if rank == 0:
+            print(json.dumps({"cgee": cgee_measurement(rk, dev, flush, measured_peak_gbs()[0], iters=max(3, args.steps))}))
+        return
+
+    w = load_workload(args.workload, seed_shift=rank)
+    batch = DeviceBatch(w, dev)
+    if w.name == "long_context":
+        punch_long_context(rk, batch)
 
     plan = None
     for _ in range(max(args.warmup, 3)):
@@ -517,6 +525,7 @@ def run_ours(args):
         if not args.no_sweep:
             line["configs"] = sweep_configs(rk, dev, flush, peak_gbs, skip=args.workload, cached=(args.workload, line))
             line["suffix_prefill"] = suffix_prefill_measurement(rk, dev, flush, args.workload, 16)
+            line["cgee"] = cgee_measurement(rk, dev, flush, peak_gbs)
         if not args.no_cpu_baseline:
             # about 10-30 s of oracle work: whole passes over the batch until 10 s have gone by
             passes, total, ub, cores, nb, Bt = 0, 0.0, 0, 1, 0, 0
@@ -697,6 +706,41 @@ def suffix_prefill_measurement(rk, dev, flush, workload: str, s: int):
     del b
     torch.cuda.empty_cache()
     return res
+
+
+def cgee_measurement(rk, dev, flush, peak_gbs, B=8, D=3584, V=152064, iters=12):
+    """The entropy hook of CGEE (Section 2.3, Eq. 5 / Algorithm 3) on Qwen2.5-7B's shapes: B = 8 verify rows,
+    D = 3584, V = 152064; synthetic W_u and hidden rows.  The kernel reads W_u once: HBM roofline on its bytes."""
+    import torch
+    import workloads
+    h, w = workloads.make_cgee_inputs(B, D, V, seed=workloads.generators.SEED_BASE + 60)
+    h, w = h.to(dev), w.to(dev)
+    H = torch.empty(B, dtype=torch.float32, device=dev)
+    P = torch.empty(B, dtype=torch.float32, device=dev)
+    ws = torch.empty(int(rk.lib().rksc_cgee_workspace_bytes()), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    times = []
+    for _ in range(iters):
+        flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        rk.rksc_cgee_logit_entropy(h, w, H, P, ws, status)
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert int(status.item()) == 0
+    Hp = torch.full((B,), float("inf"), dtype=torch.float32, device=dev)
+    flags = rk.rksc_cgee_entropy_exit(H, Hp, 2, 2, 8.0, 3.0)
+    torch.cuda.synchronize()
+    med = statistics.median(times[2:])
+    byts = V * D * 2 + B * D * 2
+    return {"what": f"rksc_cgee_logit_entropy: entropy and top-1 probability of softmax(h W_u^T), B = {B}, D = {D}, "
+                    f"V = {V} (two launches: the fused kernel and a one-block merge), cold L2",
+            "ms_median": med, "w_u_bytes": V * D * 2,
+            "roofline": {"bound": "hbm", "achieved": byts / (med * 1e-3) / 1e9, "peak": peak_gbs, "unit": "GB/s",
+                         "frac": byts / (med * 1e-3) / 1e9 / peak_gbs, "algorithmic_bytes_per_launch": byts},
+            "tflops": 2.0 * B * D * V / (med * 1e-3) / 1e12,
+            "entropy_nats_min_max": [float(H.min()), float(H.max())], "exit_flags_at_first_layer": int(flags.sum())}
 
 
 def sweep_configs(rk, dev, flush, peak_gbs, skip, cached):
