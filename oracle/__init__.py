@@ -25,6 +25,8 @@ written for reading rather than speed:
 
 * ``logit_entropy`` / ``entropy_exit`` / ``generation_confidence`` / ``verify_skip`` - the
                          numerics of CGEE (Section 2.3, Eq. 3-5, Algorithm 3).
+* ``append_token`` / ``write_token`` - one step of the token-by-token decode on the paged
+                         cache (Appendix "Stepwise Batched Decode", step 2): index work.
 
 Parity pins: every function here is pinned by the CPU tests against closed
 forms, brute force on tiny inputs and invariants; none is "parity unpinned".
@@ -40,3 +42,4 @@ from .branch_attention import branch_decode_attention, to_f32_numpy  # noqa: F40
 from .rsbcm import page_scores, rsbcm_evict, apply_eviction  # noqa: F401
 from .suffix_prefill import suffix_prefill_attention, suffix_prefill_tables  # noqa: F401
 from .cgee import logit_entropy, entropy_exit, generation_confidence, verify_skip  # noqa: F401
+from .decode_loop import append_token, write_token  # noqa: F401
