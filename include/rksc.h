@@ -378,6 +378,30 @@ RKSC_API int32_t rksc_cgee_entropy_exit(const float* entropy, const float* entro
 RKSC_API int32_t rksc_cgee_verify_skip(const float* top1_per_step, int32_t t, int32_t B, float tau_conf,
                                        float r_gap, float* confidence, int32_t* skip, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Token-by-token decode on the paged cache (paper Appendix "Stepwise Batched Decode", step (2)).
+ * One decode step = rksc_tables_append_token (host: where each branch's new token goes, and the
+ * tables afterwards), rksc_kv_append (device: the new keys and values into the pool), then a plan
+ * from the new tables and rksc_branch_decode_attention as for any step.
+ *
+ * rksc_tables_append_token: every branch that lists segments gains one token at the end of its
+ * last segment, which no other branch (and no other position of that branch) may list - its
+ * private suffix.  When that segment's pages are full (or it has none) page new_pages[b] is
+ * appended to it first (new_pages may be NULL if no branch needs one).  page[b], slot[b] (host
+ * arrays [B], out) say where branch b's token is stored: k_pool[page][kvh][slot][:]; -1, -1 for
+ * a branch without segments.  `out` is allocated by the library (rksc_tables_free).
+ * Errors: RKSC_ERR_INVALID_ARG (NULL arguments, a needed new page missing or negative),
+ * RKSC_ERR_BAD_TABLE (inconsistent tables, a shared last segment), RKSC_ERR_NOMEM.
+ *
+ * rksc_kv_append: k_pool[page[b]][h][slot[b]][:] = k_new[b][h][:] (v likewise) for every branch
+ * with page[b] >= 0; entries outside the pool are skipped.  Device pointers: pools as for the
+ * attention, k_new / v_new bf16 [B][Hkv][d], page / slot int32 [B]; all 16-byte aligned.
+ * ------------------------------------------------------------------------------------------ */
+RKSC_API int32_t rksc_tables_append_token(const rksc_tables* in, const int32_t* new_pages, rksc_tables* out,
+                                          int32_t* page, int32_t* slot);
+RKSC_API int32_t rksc_kv_append(const rksc_layout* layout, void* k_pool, void* v_pool, const void* k_new,
+                                const void* v_new, int32_t B, const int32_t* page, const int32_t* slot, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

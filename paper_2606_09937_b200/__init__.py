@@ -27,6 +27,8 @@ from .binding import (  # noqa: F401
     rksc_rsbcm_evict,
     rksc_tables_drop_evicted,
     rksc_tables_for_suffix_prefill,
+    rksc_tables_append_token,
+    rksc_kv_append,
     rksc_cgee_logit_entropy,
     rksc_cgee_entropy_exit,
     rksc_cgee_verify_skip,

@@ -36,6 +36,8 @@ EXPORTED_SYMBOLS = (
     "rksc_rsbcm_evict",
     "rksc_tables_drop_evicted",
     "rksc_tables_for_suffix_prefill",
+    "rksc_tables_append_token",
+    "rksc_kv_append",
     "rksc_cgee_workspace_bytes",
     "rksc_cgee_logit_entropy",
     "rksc_cgee_entropy_exit",
@@ -126,6 +128,10 @@ def lib() -> C.CDLL:
     L.rksc_rsbcm_evict.restype = C.c_int32
     L.rksc_rsbcm_evict.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_size_t, C.c_void_p]
+    L.rksc_tables_append_token.restype = C.c_int32
+    L.rksc_tables_append_token.argtypes = [C.POINTER(_CTables), i32p, C.POINTER(_CTables), i32p, i32p]
+    L.rksc_kv_append.restype = C.c_int32
+    L.rksc_kv_append.argtypes = [C.POINTER(_CLayout)] + [C.c_void_p] * 4 + [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     L.rksc_cgee_workspace_bytes.restype = C.c_size_t
     L.rksc_cgee_workspace_bytes.argtypes = []
     L.rksc_cgee_logit_entropy.restype = C.c_int32
@@ -453,6 +459,37 @@ def rksc_tables_drop_evicted(tables, evicted) -> Tables:
     finally:
         lib().rksc_tables_free(C.byref(out))
     return res
+
+
+def rksc_tables_append_token(tables, new_pages):
+    """Host call: one decode step on the tables.  Returns (Tables, page int32 [B], slot int32 [B])."""
+    t = Tables.of(tables)
+    B = len(t.br_seg_off) - 1
+    npg = _i32(new_pages) if new_pages is not None else None
+    page = np.empty(max(B, 1), dtype=np.int32)
+    slot = np.empty(max(B, 1), dtype=np.int32)
+    out = _CTables()
+    st = lib().rksc_tables_append_token(C.byref(t.c), _p(npg) if npg is not None else None, C.byref(out), _p(page), _p(slot))
+    _check(st, "rksc_tables_append_token")
+    try:
+        S = out.num_segments
+        cp = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(max(n, 1),))[:n].copy()
+        seg_block_off = cp(out.seg_block_off, S + 1)
+        br_seg_off = cp(out.br_seg_off, B + 1)
+        res = Tables(seg_block_off, cp(out.seg_blocks, int(seg_block_off[-1])), cp(out.seg_num_tokens, S),
+                     br_seg_off, cp(out.br_segs, int(br_seg_off[-1])))
+    finally:
+        lib().rksc_tables_free(C.byref(out))
+    return res, page[:B], slot[:B]
+
+
+def rksc_kv_append(layout, k_pool, v_pool, k_new, v_new, page, slot, stream=None):
+    """Device call: the new token's keys and values (bf16 [B][Hkv][d]) into the paged pools at (page, slot)
+    (device int32 [B])."""
+    lay = layout if isinstance(layout, Layout) else Layout.of(layout)
+    st = lib().rksc_kv_append(C.byref(lay.c), k_pool.data_ptr(), v_pool.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
+                              int(k_new.shape[0]), page.data_ptr(), slot.data_ptr(), _stream_ptr(stream, k_pool.device))
+    _check(st, "rksc_kv_append")
 
 
 def rksc_cgee_logit_entropy(h, w_u, entropy=None, top1_prob=None, workspace=None, device_status=None, stream=None):

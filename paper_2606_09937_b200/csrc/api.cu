@@ -741,3 +741,28 @@ extern "C" RKSC_API int32_t rksc_cgee_verify_skip(const float* top1_per_step, in
     }
     return RKSC_OK;
 }
+
+// ---- token-by-token decode on the paged cache (Appendix "Stepwise Batched Decode", step 2) ----
+
+extern "C" RKSC_API int32_t rksc_kv_append(const rksc_layout* layout, void* k_pool, void* v_pool, const void* k_new,
+                                           const void* v_new, int32_t B, const int32_t* page, const int32_t* slot,
+                                           void* stream) {
+    if (!layout || B < 0) return RKSC_ERR_INVALID_ARG;
+    if (B == 0) return RKSC_OK;
+    if (!k_pool || !v_pool || !k_new || !v_new || !page || !slot) return RKSC_ERR_INVALID_ARG;
+    if (layout->num_kv_heads <= 0 || layout->head_dim <= 0 || layout->num_pool_blocks <= 0) return RKSC_ERR_INVALID_ARG;
+    if (layout->block_size != kBlock) return RKSC_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(k_pool) & 15) || (reinterpret_cast<uintptr_t>(v_pool) & 15) ||
+        (reinterpret_cast<uintptr_t>(k_new) & 15) || (reinterpret_cast<uintptr_t>(v_new) & 15))
+        return RKSC_ERR_INVALID_ARG;
+    int32_t st = ensure_device(nullptr);
+    if (st != RKSC_OK) return st;
+    cudaError_t e = launch_kv_append(k_pool, v_pool, k_new, v_new, page, slot, B, layout->num_kv_heads, layout->head_dim,
+                                     layout->num_pool_blocks, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda = e;
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    return RKSC_OK;
+}

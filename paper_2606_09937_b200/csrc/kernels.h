@@ -58,6 +58,8 @@ cudaError_t launch_entropy_exit(const float* H, const float* H_prev, int B, int 
                                 int32_t* flags, cudaStream_t stream);
 cudaError_t launch_verify_skip(const float* top1_steps, int t, int B, float tau_conf, float r_gap, float* p_out,
                                int32_t* skip, cudaStream_t stream);
+cudaError_t launch_kv_append(void* k_pool, void* v_pool, const void* k_new, const void* v_new, const int32_t* page,
+                             const int32_t* slot, int B, int Hkv, int head_dim, int num_pool_blocks, cudaStream_t stream);
 cudaError_t launch_rsbcm_select(const double* score, const int32_t* depth, int32_t n, uint32_t k, uint64_t* keys,
                                 uint8_t* evicted, int32_t* num_evicted, cudaStream_t stream);
 

@@ -500,3 +500,88 @@ extern "C" RKSC_API int32_t rksc_tables_for_suffix_prefill(const rksc_tables* in
     out->br_segs = a4;
     return RKSC_OK;
 }
+
+// One decode step on the tables (Appendix "Stepwise Batched Decode", step 2): every branch with
+// segments gains a token at the end of its last segment, which it must list alone.
+extern "C" RKSC_API int32_t rksc_tables_append_token(const rksc_tables* in, const int32_t* new_pages, rksc_tables* out,
+                                                     int32_t* page, int32_t* slot) {
+    if (!in || !out) return RKSC_ERR_INVALID_ARG;
+    std::memset(out, 0, sizeof(*out));
+    const int B = in->num_branches, S = in->num_segments;
+    if (B < 0 || S < 0 || !in->seg_block_off || !in->br_seg_off) return RKSC_ERR_INVALID_ARG;
+    if (B > 0 && (!page || !slot)) return RKSC_ERR_INVALID_ARG;
+    if (S > 0 && !in->seg_num_tokens) return RKSC_ERR_INVALID_ARG;
+    if (in->seg_block_off[0] != 0 || in->br_seg_off[0] != 0) return RKSC_ERR_BAD_TABLE;
+    const int64_t N = in->seg_block_off[S], R = in->br_seg_off[B];
+    if ((N > 0 && !in->seg_blocks) || (R > 0 && !in->br_segs)) return RKSC_ERR_INVALID_ARG;
+    std::vector<int32_t> refs, grow;
+    try {
+        refs.assign((size_t)S, 0);
+        grow.assign((size_t)S, -1);   // page appended to the segment, or -1
+    } catch (const std::bad_alloc&) {
+        return RKSC_ERR_NOMEM;
+    }
+    for (int64_t i = 0; i < R; ++i) {
+        if (in->br_segs[i] < 0 || in->br_segs[i] >= S) return RKSC_ERR_BAD_TABLE;
+        refs[in->br_segs[i]]++;
+    }
+    for (int s = 0; s < S; ++s) {
+        const int64_t n = (int64_t)in->seg_block_off[s + 1] - in->seg_block_off[s];
+        const int64_t nt = in->seg_num_tokens[s];
+        if (n < 0 || nt < 0 || nt > n * rksc::kBlock || (n > 0 && nt <= (n - 1) * rksc::kBlock)) return RKSC_ERR_BAD_TABLE;
+    }
+    int64_t added = 0;
+    for (int b = 0; b < B; ++b) {
+        const int lo = in->br_seg_off[b], hi = in->br_seg_off[b + 1];
+        if (hi < lo) return RKSC_ERR_BAD_TABLE;
+        if (hi == lo) continue;
+        const int s = in->br_segs[hi - 1];
+        if (refs[s] != 1) return RKSC_ERR_BAD_TABLE;   // a shared segment cannot grow
+        const int n = in->seg_block_off[s + 1] - in->seg_block_off[s];
+        if (in->seg_num_tokens[s] == n * rksc::kBlock) {
+            if (!new_pages || new_pages[b] < 0) return RKSC_ERR_INVALID_ARG;
+            grow[s] = new_pages[b];
+            ++added;
+        }
+    }
+    if (N + added >= ((int64_t)1 << 31)) return RKSC_ERR_UNSUPPORTED;
+    auto alloc = [](size_t n) { return (int32_t*)std::malloc(std::max<size_t>(1, n) * sizeof(int32_t)); };
+    int32_t* a0 = alloc((size_t)S + 1);
+    int32_t* a1 = alloc((size_t)(N + added));
+    int32_t* a2 = alloc((size_t)S);
+    int32_t* a3 = alloc((size_t)B + 1);
+    int32_t* a4 = alloc((size_t)R);
+    if (!a0 || !a1 || !a2 || !a3 || !a4) {
+        std::free(a0); std::free(a1); std::free(a2); std::free(a3); std::free(a4);
+        return RKSC_ERR_NOMEM;
+    }
+    int32_t w = 0;
+    a0[0] = 0;
+    for (int s = 0; s < S; ++s) {
+        const int lo = in->seg_block_off[s], hi = in->seg_block_off[s + 1];
+        if (hi > lo) std::memcpy(a1 + w, in->seg_blocks + lo, (size_t)(hi - lo) * sizeof(int32_t));
+        w += hi - lo;
+        if (grow[s] >= 0) a1[w++] = grow[s];
+        a0[s + 1] = w;
+        a2[s] = in->seg_num_tokens[s];
+    }
+    for (int b = 0; b < B; ++b) {
+        const int lo = in->br_seg_off[b], hi = in->br_seg_off[b + 1];
+        page[b] = slot[b] = -1;
+        if (hi == lo) continue;
+        const int s = in->br_segs[hi - 1];
+        page[b] = a1[a0[s + 1] - 1];
+        slot[b] = a2[s] % rksc::kBlock;
+        a2[s] += 1;
+    }
+    std::memcpy(a3, in->br_seg_off, ((size_t)B + 1) * sizeof(int32_t));
+    if (R > 0) std::memcpy(a4, in->br_segs, (size_t)R * sizeof(int32_t));
+    out->num_branches = B;
+    out->num_segments = S;
+    out->seg_block_off = a0;
+    out->seg_blocks = a1;
+    out->seg_num_tokens = a2;
+    out->br_seg_off = a3;
+    out->br_segs = a4;
+    return RKSC_OK;
+}

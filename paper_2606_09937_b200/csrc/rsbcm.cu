@@ -215,3 +215,42 @@ cudaError_t launch_rsbcm_select(const double* score, const int32_t* depth, int32
 }
 
 }  // namespace rksc
+
+// ---- token-by-token decode: the new token's key and value into the paged pool ----
+namespace rksc {
+namespace {
+// One warp per (branch, KV head): copies d bf16 of K and of V (16-byte pieces when d allows).
+__global__ void kv_append_kernel(uint8_t* __restrict__ k_pool, uint8_t* __restrict__ v_pool, const uint8_t* __restrict__ k_new,
+                                 const uint8_t* __restrict__ v_new, const int32_t* __restrict__ page,
+                                 const int32_t* __restrict__ slot, int B, int Hkv, int row_bytes, int num_pool_blocks) {
+    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (gw >= B * Hkv) return;
+    const int b = gw / Hkv, h = gw % Hkv;
+    const int pg = page[b], sl = slot[b];
+    if (pg < 0 || pg >= num_pool_blocks || sl < 0 || sl >= kBlock) return;   // no token for this branch (or a bad entry: skipped)
+    const size_t dst = (((size_t)pg * Hkv + h) * kBlock + sl) * row_bytes;
+    const size_t src = ((size_t)b * Hkv + h) * row_bytes;
+    if ((row_bytes & 15) == 0) {
+        for (int i = lane * 16; i < row_bytes; i += 32 * 16) {
+            *reinterpret_cast<uint4*>(k_pool + dst + i) = *reinterpret_cast<const uint4*>(k_new + src + i);
+            *reinterpret_cast<uint4*>(v_pool + dst + i) = *reinterpret_cast<const uint4*>(v_new + src + i);
+        }
+    } else {
+        for (int i = lane * 2; i < row_bytes; i += 64) {
+            *reinterpret_cast<uint16_t*>(k_pool + dst + i) = *reinterpret_cast<const uint16_t*>(k_new + src + i);
+            *reinterpret_cast<uint16_t*>(v_pool + dst + i) = *reinterpret_cast<const uint16_t*>(v_new + src + i);
+        }
+    }
+}
+}  // namespace
+
+cudaError_t launch_kv_append(void* k_pool, void* v_pool, const void* k_new, const void* v_new, const int32_t* page,
+                             const int32_t* slot, int B, int Hkv, int head_dim, int num_pool_blocks, cudaStream_t stream) {
+    if (B <= 0) return cudaSuccess;
+    const int warps = B * Hkv;
+    kv_append_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(static_cast<uint8_t*>(k_pool), static_cast<uint8_t*>(v_pool),
+                                                         static_cast<const uint8_t*>(k_new), static_cast<const uint8_t*>(v_new),
+                                                         page, slot, B, Hkv, head_dim * 2, num_pool_blocks);
+    return cudaGetLastError();
+}
+}  // namespace rksc
