@@ -526,6 +526,7 @@ def run_ours(args):
             line["configs"] = sweep_configs(rk, dev, flush, peak_gbs, skip=args.workload, cached=(args.workload, line))
             line["suffix_prefill"] = suffix_prefill_measurement(rk, dev, flush, args.workload, 16)
             line["cgee"] = cgee_measurement(rk, dev, flush, peak_gbs)
+            line["decode_loop"] = decode_loop_measurement(rk, dev, args.workload)
         if not args.no_cpu_baseline:
             # about 10-30 s of oracle work: whole passes over the batch until 10 s have gone by
             passes, total, ub, cores, nb, Bt = 0, 0.0, 0, 1, 0, 0
@@ -703,6 +704,79 @@ def suffix_prefill_measurement(rk, dev, flush, workload: str, s: int):
            "unique_kv_bytes_of_the_decode_tables": kv0, "tbps_on_those_bytes": kv0 / (med * 1e-3) / 1e12,
            "kv_bytes_the_plan_reads": plan.unique_kv_tokens * 2 * lay.num_kv_heads * lay.head_dim * 2,
            "attention_tflops": flops / (med * 1e-3) / 1e12, "work_items": plan.num_work_items}
+    del b
+    torch.cuda.empty_cache()
+    return res
+
+
+def decode_loop_measurement(rk, dev, workload: str, steps: int = 32):
+    """Token-by-token decode (Appendix "Stepwise Batched Decode", step 2) on a config's tables: every step
+    appends one token per branch to the paged cache (tables on the host, keys and values on the device), builds
+    the plan of the grown tables and runs the attention.  Strictly serial steps (each needs the previous token)."""
+    import dataclasses
+    import torch
+    w = load_workload(workload)
+    b = DeviceBatch(w, dev)
+    run_step(rk, b)
+    torch.cuda.synchronize()
+    if b.has_gate:
+        f = w.flat
+        t = rk.rksc_tables_from_gate(b.map_host.numpy(), f.num_prefixes, f.shared_off, f.shared_pages, f.shared_ntok,
+                                     f.priv_off, f.priv_pages, f.priv_ntok, f.sfx_off, f.sfx_pages, f.sfx_ntok)
+    else:
+        t = b.tables
+    B, Hq, d = b.q.shape
+    lay0 = w.layout
+    extra = B * (steps // 16 + 2)
+    nblk = lay0.num_pool_blocks
+    grow = lambda p: torch.cat([p, torch.zeros((extra,) + tuple(p.shape[1:]), dtype=p.dtype, device=dev)])
+    k_pool, v_pool = grow(b.k_pool), grow(b.v_pool)
+    b.k_pool = b.v_pool = None
+    lay = rk.Layout.of(dataclasses.replace(lay0, num_pool_blocks=nblk + extra))
+    g = torch.Generator(device="cpu").manual_seed(77)
+    k_new = torch.randn((B, lay0.num_kv_heads, d), generator=g).to(torch.bfloat16).to(dev)
+    v_new = torch.randn((B, lay0.num_kv_heads, d), generator=g).to(torch.bfloat16).to(dev)
+    page_dev = torch.empty(B, dtype=torch.int32, device=dev)
+    slot_dev = torch.empty(B, dtype=torch.int32, device=dev)
+    page_host = torch.empty(B, dtype=torch.int32).pin_memory()
+    slot_host = torch.empty(B, dtype=torch.int32).pin_memory()
+    new_pages = np.arange(nblk, nblk + B, dtype=np.int32)      # one spare page per branch per 16 steps
+    plan = rk.rksc_plan_create(lay, t)
+    out = torch.empty((B, Hq, d), dtype=torch.float32, device=dev)
+    mass = torch.empty(max(plan.mass_elems, 1) + B * Hq * (steps // 16 + 2), dtype=torch.float32, device=dev)
+    ws = torch.empty(2 * plan.workspace_bytes, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def one(step, t):
+        t, page, slot = rk.rksc_tables_append_token(t, new_pages + B * (step // 16))
+        page_host.copy_(torch.from_numpy(page))
+        slot_host.copy_(torch.from_numpy(slot))
+        page_dev.copy_(page_host, non_blocking=True)
+        slot_dev.copy_(slot_host, non_blocking=True)
+        rk.rksc_kv_append(lay, k_pool, v_pool, k_new, v_new, page_dev, slot_dev)
+        plan = rk.rksc_plan_create(lay, t)
+        assert plan.workspace_bytes <= ws.numel() and plan.mass_elems <= mass.numel()
+        rk.rksc_branch_decode_attention(plan, b.q, k_pool, v_pool, out=out, block_mass=mass, workspace=ws,
+                                        device_status=status)
+        return t, plan
+
+    for step in range(3):                                    # warm-up steps (they grow the tables too)
+        t, plan = one(step, t)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    for step in range(3, 3 + steps):
+        t, plan = one(step, t)
+    e1.record()
+    e1.synchronize()
+    wall = time.perf_counter() - t0
+    assert int(status.item()) == 0
+    ms = e0.elapsed_time(e1) / steps
+    res = {"what": f"{steps} serial decode steps on {workload}: tables append (host) + keys/values append (device) + "
+                   "plan of the grown tables + attention, one new token per branch and step",
+           "ms_per_step": ms, "wall_ms_per_step": wall * 1e3 / steps, "tokens_per_s": B / (ms * 1e-3),
+           "branches": B}
     del b
     torch.cuda.empty_cache()
     return res
