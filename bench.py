@@ -63,6 +63,8 @@ def parse_args():
     ap.add_argument("--no-pipeline", action="store_true", help="time the steps strictly one after another")
     ap.add_argument("--cgee-only", action="store_true",
                     help="run only the CGEE entropy-kernel measurement and print its object (used for profiling)")
+    ap.add_argument("--model-step-only", action="store_true",
+                    help="run only the whole-model decode-step measurement (all layers, eager and as a CUDA graph)")
     return ap.parse_args()
 
 
@@ -403,6 +405,11 @@ def run_ours(args):
             print(json.dumps({"cgee": cgee_measurement(rk, dev, flush, measured_peak_gbs()[0], iters=max(3, args.steps))}))
         return
 
+    if args.model_step_only:
+        if rank == 0:
+            print(json.dumps({"model_step": model_step_measurement(rk, dev, args.workload)}))
+        return
+
     w = load_workload(args.workload, seed_shift=rank)
     batch = DeviceBatch(w, dev)
     if w.name == "long_context":
@@ -527,6 +534,7 @@ def run_ours(args):
             line["suffix_prefill"] = suffix_prefill_measurement(rk, dev, flush, args.workload, 16)
             line["cgee"] = cgee_measurement(rk, dev, flush, peak_gbs)
             line["decode_loop"] = decode_loop_measurement(rk, dev, args.workload)
+            line["model_step"] = model_step_measurement(rk, dev, args.workload)
         if not args.no_cpu_baseline:
             # about 10-30 s of oracle work: whole passes over the batch until 10 s have gone by
             passes, total, ub, cores, nb, Bt = 0, 0.0, 0, 1, 0, 0
@@ -778,6 +786,74 @@ def decode_loop_measurement(rk, dev, workload: str, steps: int = 32):
            "ms_per_step": ms, "wall_ms_per_step": wall * 1e3 / steps, "tokens_per_s": B / (ms * 1e-3),
            "branches": B}
     del b
+    torch.cuda.empty_cache()
+    return res
+
+
+def model_step_measurement(rk, dev, workload: str, layers: int = 28, iters: int = 5):
+    """One decode step of a whole model: the attention of every layer, each layer on its own KV pool, all through
+    the step's one plan (Appendix "Stepwise Batched Decode": the tables are the step's, not the layer's).  Timed
+    twice: the calls enqueued one by one, and the same calls captured once in a CUDA graph and replayed.  The
+    layers' pools together are far larger than L2, so every layer reads cold."""
+    import dataclasses
+    import torch
+    import workloads
+    w = load_workload(workload)
+    b = DeviceBatch(w, dev)
+    plan, _ = run_step(rk, b)
+    torch.cuda.synchronize()
+    B, Hq, d = b.q.shape
+    kv_bytes, _ = algorithmic_bytes(plan, w.layout)
+    base = dataclasses.replace(w, q=b.q, k_pool=b.k_pool, v_pool=b.v_pool)
+    per_layer = [workloads.layer_variant(base, l) for l in range(layers)]
+    outs = [torch.empty((B, Hq, d), dtype=torch.float32, device=dev) for _ in range(layers)]
+    masses = [torch.empty(max(plan.mass_elems, 1), dtype=torch.float32, device=dev) for _ in range(layers)]
+    ws = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def enqueue():
+        for l, x in enumerate(per_layer):
+            rk.rksc_branch_decode_attention(plan, x.q, x.k_pool, x.v_pool, out=outs[l], block_mass=masses[l],
+                                            workspace=ws, device_status=status)
+
+    def timed(fn):
+        times, walls = [], []
+        for _ in range(iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            e0.record()
+            fn()
+            walls.append(time.perf_counter() - t0)
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+        return statistics.median(times), statistics.median(walls) * 1e3
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            enqueue()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    eager_ms, eager_cpu_ms = timed(enqueue)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        enqueue()
+    graph.replay()
+    torch.cuda.synchronize()
+    graph_ms, graph_cpu_ms = timed(graph.replay)
+    assert int(status.item()) == 0
+    res = {"what": f"attention of {layers} layers of one decode step on {workload} (one plan, one pool per layer, "
+                   f"{layers * kv_bytes / 1e9:.1f} GB of unique KV in all): enqueued call by call, and as one CUDA graph",
+           "layers": layers, "graph_ms_per_step": graph_ms, "eager_ms_per_step": eager_ms,
+           "graph_us_per_layer": graph_ms * 1e3 / layers,
+           "graph_enqueue_cpu_ms": graph_cpu_ms, "eager_enqueue_cpu_ms": eager_cpu_ms,
+           "tbps_unique_kv": layers * kv_bytes / (graph_ms * 1e-3) / 1e12,
+           "pct_of_8tbps": 100.0 * layers * kv_bytes / (graph_ms * 1e-3) / 1e12 / NOMINAL_HBM_TBPS,
+           "whole_model_branch_steps_per_s": B / (graph_ms * 1e-3)}
+    del graph, per_layer, outs, masses, b
     torch.cuda.empty_cache()
     return res
 

@@ -27,6 +27,7 @@ from .generators import (  # noqa: F401
     make_block_masses,
     make_eviction_inputs,
     make_cgee_inputs,
+    layer_variant,
     unique_kv_bytes,
     duplicated_kv_bytes,
     CONFIG_NAMES,

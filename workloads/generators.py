@@ -458,6 +458,22 @@ def make_cgee_inputs(B: int, D: int, V: int, seed: int = SEED_BASE + 60, logit_s
     return h.to(torch.bfloat16), w.to(torch.bfloat16)
 
 
+def layer_variant(w: Workload, layer: int) -> Workload:
+    """The inputs of another transformer layer of the same decode step: the tables (and so the page
+    ids, token counts and sharing) are the step's, the numbers are the layer's own.  Layer 0 is ``w``;
+    layer l > 0 holds w's values moved around - keys rotated by l along head_dim, values by 3 l + 1,
+    queries by l along the branch axis - so that every layer has a different result while the
+    sentinel in the unused slots of partial pages stays where it is.  Works on host or device tensors."""
+    if layer == 0:
+        return w
+    d = w.layout.head_dim
+    return dataclasses.replace(
+        w, name=f"{w.name}/layer{layer}",
+        q=torch.roll(w.q, shifts=layer, dims=0).contiguous(),
+        k_pool=torch.roll(w.k_pool, shifts=layer % d, dims=-1).contiguous(),
+        v_pool=torch.roll(w.v_pool, shifts=(3 * layer + 1) % d, dims=-1).contiguous())
+
+
 def make_config(name: str, **kw) -> Workload:
     if name == "tiny":
         return make_tiny(**kw)
