@@ -45,6 +45,9 @@ WORKLOAD_LABEL = {
                        "suffix U[128,1024], 28q/4kv d128, 30% of branches below tau",
     "long_context": "configs[4] long context with eviction holes: 16 branches, prefix 32768 (20% of pages "
                     "evicted) + suffix 2048, 32q/8kv d128",
+    "diverse_phrasing": "diverse-phrasing regime (not a BASELINE config): 15 problems x 8 phrasings at 4 divergence "
+                        "levels, prefix 512, suffix U[16,144], 28q/4kv d128, alpha 1.5, tau 0.82; the gate shares "
+                        "the identical and the minor-rewording phrasings",
 }
 
 
@@ -141,7 +144,8 @@ class ClockSampler:
 
 def load_workload(name: str, seed_shift: int = 0):
     import workloads
-    base = {"tiny": 0, "qwen_layer": 1, "tot": 2, "batched_serving": 3, "long_context": 4}[name]
+    base = {"tiny": 0, "qwen_layer": 1, "tot": 2, "batched_serving": 3, "long_context": 4,
+            "diverse_phrasing": 5}[name]
     return workloads.make_config(name, seed=workloads.generators.SEED_BASE + base + 1000 * seed_shift)
 
 
@@ -915,6 +919,12 @@ def sweep_configs(rk, dev, flush, peak_gbs, skip, cached):
                      "tbps_unique_kv": kv / (med * 1e-3) / 1e12,
                      "pct_of_8tbps": 100.0 * kv / (med * 1e-3) / 1e12 / NOMINAL_HBM_TBPS,
                      "branch_steps_per_s": b.w.num_branches / (med * 1e-3), "work_items": plan.num_work_items}
+        if name == "diverse_phrasing":
+            shared = (b.map_host.numpy() >= 0)
+            nonroot = np.arange(shared.size) % 8 != 0
+            res[name]["gate_shares_of_non_root_phrasings"] = float(shared[nonroot].mean())
+            res[name]["exact_token_cache_would_share"] = float((b.w.phrasing_level == 0)[nonroot].mean())
+            res[name]["duplicated_over_unique_kv"] = plan.duplicated_kv_tokens / max(plan.unique_kv_tokens, 1)
         if rsbcm is not None:
             res[name]["rsbcm_eviction_before_this_step"] = rsbcm
         del b

@@ -22,6 +22,7 @@ from .generators import (  # noqa: F401
     make_tot,
     make_batched_serving,
     make_long_context,
+    make_diverse_phrasing,
     punch_holes,
     lowest_mass_pages,
     make_block_masses,

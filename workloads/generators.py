@@ -112,6 +112,7 @@ class Workload:
     flat: Optional[FlatLists] = None  # two-level lists, when tables come from the gate
     gate: Optional[GateInputs] = None
     notes: str = ""
+    phrasing_level: Optional[np.ndarray] = None   # diverse-phrasing regime: divergence level of each branch
 
     @property
     def num_branches(self) -> int:
@@ -378,6 +379,42 @@ def make_long_context(seed: int = SEED_BASE + 4, prefix: int = 32768, suffix: in
     return w
 
 
+# eps of the four semantic-divergence levels of the diverse-phrasing regime (cos = 1 / sqrt(1 + eps^2)):
+# identical 1.0, minor rewording 0.94, structural reframing 0.74, very different register 0.45
+PHRASING_EPS = (0.0, 0.35, 0.9, 2.0)
+
+
+def make_diverse_phrasing(seed: int = SEED_BASE + 5, problems: int = 15, templates: int = 8,
+                          prefix: int = 512, sfx_lo: int = 16, sfx_hi: int = 144,
+                          num_q_heads: int = 28, num_kv_heads: int = 4, head_dim: int = 128,
+                          L: int = 28, D: int = 3584) -> Workload:
+    """The diverse-phrasing regime of Section "ASKS Novelty Over vLLM Prefix Caching": every problem is
+    posed through ``templates`` phrasings spread evenly over four semantic-divergence levels, padded to
+    about ``prefix`` tokens; phrasing 0 is the problem's root.  Qwen2.5-7B shapes, the paper's default
+    alpha = 1.5 and tau = 0.82.  The hidden states of a phrasing sit at the angle of its level from the
+    root's (PHRASING_EPS), so the two closer levels pass the gate and the two farther ones keep a
+    private prefix.  Tables come from the gate map (end to end, like the batched-serving config).
+
+    ``w.notes`` records which branches an exact-token prefix cache could share (level 0 only)."""
+    assert templates % 4 == 0
+    per_level = templates // 4
+    B = problems * templates
+    rng = np.random.default_rng([SEED_BASE, int(seed), 13])
+    level = np.array([(b % templates) // per_level for b in range(B)], dtype=np.int32)
+    branch_problem = [b // templates for b in range(B)]
+    sfx_ntok = rng.integers(sfx_lo, sfx_hi + 1, size=B)
+    far = np.flatnonzero(level >= 2)
+    w = _two_level("diverse_phrasing", num_q_heads, num_kv_heads, head_dim, [prefix] * problems,
+                   branch_problem, far.tolist(), sfx_ntok.tolist(), seed)
+    eps = [PHRASING_EPS[int(l)] for l in level]
+    w.gate = make_gate_inputs(branch_problem, problems, L, D, eps, alpha=1.5, tau=0.82, seed=seed)
+    w.tables = None
+    w.phrasing_level = level
+    w.notes = (f"{problems} problems x {templates} phrasings at 4 divergence levels; an exact-token cache "
+               f"shares level 0 only, the gate is built to share levels 0 and 1")
+    return w
+
+
 def lowest_mass_pages(scores: np.ndarray, frac: float = 0.2) -> np.ndarray:
     """Logical indices of the floor(frac*n) pages with the lowest score (ties: lower index)."""
     scores = np.asarray(scores, dtype=np.float64)
@@ -485,6 +522,8 @@ def make_config(name: str, **kw) -> Workload:
         return make_batched_serving(**kw)
     if name == "long_context":
         return make_long_context(**kw)
+    if name == "diverse_phrasing":
+        return make_diverse_phrasing(**kw)
     raise ValueError(f"unknown config {name!r}; choose from {CONFIG_NAMES}")
 
 
