@@ -151,10 +151,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (clock64() - t0 > (1ll << 32)) return false;
     }
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+// Keys and values are read once per launch: their lines are marked first to leave L2, so that the
+// partial results and block masses written meanwhile are still there when the merge reads them.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar,
+                                            uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar), "l"(policy)
         : "memory");
 }
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -380,6 +389,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         // K and V travel in rings of their own, each fed by its own warp (one warp cannot issue TMA
         // copies fast enough for the whole stream): K of a slot is needed two slots before its softmax
         // starts and is free again as soon as Q K^T has run, V is needed after the softmax.
+        const uint64_t kv_policy = l2_evict_first_policy();
         int seq = 0;
         int idx = (int)blockIdx.x;
         WorkItem it = fetch_item(idx);
@@ -405,7 +415,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 __syncwarp();
                 if (lane < npg * 2) {
                     const int y = (page * a.Hkv + it.kv_head) * kBlock;
-                    tma_load_2d(sbase + kslot * kKBytes + (lane >> 1) * 2048 + (lane & 1) * 8192, &tm_k, (lane & 1) * 64, y, full);
+                    tma_load_2d(sbase + kslot * kKBytes + (lane >> 1) * 2048 + (lane & 1) * 8192, &tm_k, (lane & 1) * 64, y, full, kv_policy);
                 }
             }
             idx = nidx;
@@ -430,6 +440,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const int bfull = kBarFullV, bempty = kBarEmptyV;
         const uint32_t ring = sbase + kVOff;
         const CUtensorMap* tm = &tm_v;
+        const uint64_t kv_policy = l2_evict_first_policy();
         int seq = 0;
         for (int k = 0; !*s_abort; ++k) {
             const int e = k % kNI;
@@ -459,7 +470,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 __syncwarp();
                 if (lane < npg * 2) {
                     const int y = (page * a.Hkv + kvh) * kBlock;
-                    tma_load_2d(ring + slot * kKBytes + (lane >> 1) * 2048 + (lane & 1) * 8192, tm, (lane & 1) * 64, y, full);
+                    tma_load_2d(ring + slot * kKBytes + (lane >> 1) * 2048 + (lane & 1) * 8192, tm, (lane & 1) * 64, y, full, kv_policy);
                 }
             }
         }

@@ -92,10 +92,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (clock64() - t0 > (1ll << 32)) return false;
     }
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+// Keys and values are read once per launch: their lines are marked first to leave L2, so that the
+// partial results and block masses written meanwhile are still there when the merge reads them.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar,
+                                            uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar), "l"(policy)
         : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
@@ -242,6 +251,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         auto fetch_ids = [&](const WorkItem& w, int first) {   // page ids first + lane of the item (0 past its end)
             return (first + lane < w.num_pages) ? __ldg(a.plan.seg_blocks + w.page_begin + first + lane) : 0;
         };
+        const uint64_t kv_policy = l2_evict_first_policy();
         int seq = 0;
         int idx = claim();
         WorkItem it = fetch_item(idx);
@@ -287,7 +297,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     const int y = (page * a.Hkv + it.kv_head) * kBlock;
                     const uint32_t dst = ring + slot * SL::kSlot + lane * SL::kPage;
 #pragma unroll
-                    for (int hh = 0; hh < HD / 64; ++hh) tma_load_2d(dst + hh * 2048, &tm_k, hh * 64, y, bar);
+                    for (int hh = 0; hh < HD / 64; ++hh) tma_load_2d(dst + hh * 2048, &tm_k, hh * 64, y, bar, kv_policy);
                 }
             }
             idx = nidx;
@@ -328,6 +338,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         // One warp cannot issue TMA copies fast enough for a CTA's share of the memory bandwidth: this
         // one follows the K producer slot by slot (header and page ids through shared memory) and
         // issues the V half of every slot.
+        const uint64_t kv_policy = l2_evict_first_policy();
         for (int seq = 0; !*s_abort; ++seq) {
             const int slot = seq % kNS;
             wait_or_abort(bar_hdr + 8 * slot, (uint32_t)(seq / kNS) & 1u);
@@ -348,7 +359,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 const int y = (page * a.Hkv + kvh) * kBlock;
                 const uint32_t dst = ring + slot * SL::kSlot + lane * SL::kPage + SL::kTile;
 #pragma unroll
-                for (int hh = 0; hh < HD / 64; ++hh) tma_load_2d(dst + hh * 2048, &tm_v, hh * 64, y, bar);
+                for (int hh = 0; hh < HD / 64; ++hh) tma_load_2d(dst + hh * 2048, &tm_v, hh * 64, y, bar, kv_policy);
             }
         }
         return;

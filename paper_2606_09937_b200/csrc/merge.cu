@@ -29,6 +29,9 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+constexpr int kPartBatch = 8;   // partial rows a lane has in flight at once
+constexpr int kMassBatch = 8;   // block masses a lane has in flight at once
+
 __global__ void __launch_bounds__(kMergeThreads)
 merge_kernel(const AttnArgs a, const int wpk_log2) {
     const int lane = threadIdx.x & 31;
@@ -36,74 +39,105 @@ merge_kernel(const AttnArgs a, const int wpk_log2) {
     const int bh = gw >> wpk_log2;
     const int sub = gw & ((1 << wpk_log2) - 1), wpk = 1 << wpk_log2;
     const bool live = bh < a.B * a.Hq;
-    int b = 0, h = 0, lo = 0, hi = 0;
+    int b = 0, h = 0, lo = 0, hi = 0, nblk = 0;
+    float* mass = nullptr;
     if (live) {
         b = bh / a.Hq;
         h = bh % a.Hq;
         const int key = b * a.Hkv + h / a.G;
         lo = a.plan.merge_off[key];
         hi = a.plan.merge_off[key + 1];
+        if (a.block_mass != nullptr && hi > lo) {
+            nblk = a.plan.br_nblk[b];
+            mass = a.block_mass + a.plan.mass_off[b] * a.Hq + (int64_t)h * nblk;
+        }
     }
     const int gi = h % a.G;
     const int HD = a.head_dim;
     // the first 32 part rows of this warp's list (plan data: readable before the dependency resolves)
-    int row_l = (lo + lane < hi) ? a.plan.merge_rows[lo + lane] + gi : -1;
+    const int row_l = (lo + lane < hi) ? a.plan.merge_rows[lo + lane] + gi : -1;
 
     // everything below reads what the segment kernel wrote
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (!live) return;
 
-    // LSE over the parts
-    float mx = -INFINITY;
-    for (int i = lo + lane; i < hi; i += 32) {
-        const int row = (i < lo + 32) ? row_l : a.plan.merge_rows[i] + gi;
-        mx = fmaxf(mx, a.part_lse[row]);
+    // Everything this warp needs is fetched with as few dependent round trips to L2 as possible: the
+    // log-sum-exps of the parts, the first batch of partial rows and the first batch of block masses
+    // are all requested before anything is reduced.
+    const bool has_cols = (4 * lane < HD) && sub == 0;
+    const float my_lse = (row_l >= 0) ? a.part_lse[row_l] : -INFINITY;
+    const int n0 = min(32, hi - lo);
+    float4 v[kPartBatch];
+#pragma unroll
+    for (int j = 0; j < kPartBatch; ++j) {
+        const int row = __shfl_sync(0xffffffffu, row_l, j);
+        v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (has_cols && j < n0) v[j] = *reinterpret_cast<const float4*>(a.part_o + (size_t)row * HD + 4 * lane);
     }
+    const int stride = 32 * wpk;
+    float mv[kMassBatch];
+#pragma unroll
+    for (int k = 0; k < kMassBatch; ++k) {
+        const int j = sub * 32 + lane + k * stride;
+        mv[k] = (j < nblk) ? mass[j] : 0.f;
+    }
+
+    // LSE over the parts
+    float mx = my_lse;
+    for (int i = lo + 32 + lane; i < hi; i += 32) mx = fmaxf(mx, a.part_lse[a.plan.merge_rows[i] + gi]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float sum = 0.f;
-    for (int i = lo + lane; i < hi; i += 32) {
-        const int row = (i < lo + 32) ? row_l : a.plan.merge_rows[i] + gi;
-        sum += fast_exp2(a.part_lse[row] - mx);
-    }
+    float sum = (row_l >= 0) ? fast_exp2(my_lse - mx) : 0.f;
+    for (int i = lo + 32 + lane; i < hi; i += 32) sum += fast_exp2(a.part_lse[a.plan.merge_rows[i] + gi] - mx);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     const float lse = mx + log2f(sum);
 
     // out (first warp of the pair): lane owns columns 4*lane .. 4*lane+3
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    const bool has_cols = (4 * lane < HD) && sub == 0;
-    for (int i0 = lo; i0 < hi && sub == 0; i0 += 32) {
-        const int n = min(32, hi - i0);
-        const int my_row = (i0 == lo) ? row_l : ((i0 + lane < hi) ? a.plan.merge_rows[i0 + lane] + gi : -1);
-        const float my_w = (my_row >= 0) ? fast_exp2(a.part_lse[my_row] - lse) : 0.f;
-        for (int j = 0; j < n; ++j) {
-            const int row = __shfl_sync(0xffffffffu, my_row, j);
-            const float w = __shfl_sync(0xffffffffu, my_w, j);
-            if (has_cols) {
-                const float4 v = *reinterpret_cast<const float4*>(a.part_o + (size_t)row * HD + 4 * lane);
-                acc.x += w * v.x;
-                acc.y += w * v.y;
-                acc.z += w * v.z;
-                acc.w += w * v.w;
+    if (sub == 0) {
+        for (int i0 = lo; i0 < hi; i0 += 32) {
+            const int n = min(32, hi - i0);
+            const int my_row = (i0 == lo) ? row_l : ((i0 + lane < hi) ? a.plan.merge_rows[i0 + lane] + gi : -1);
+            const float my_w = (my_row < 0) ? 0.f : fast_exp2(((i0 == lo) ? my_lse : a.part_lse[my_row]) - lse);
+            for (int j0 = 0; j0 < n; j0 += kPartBatch) {
+                if (i0 != lo || j0 != 0) {   // the very first batch is already here
+#pragma unroll
+                    for (int j = 0; j < kPartBatch; ++j) {
+                        const int row = __shfl_sync(0xffffffffu, my_row, (j0 + j) & 31);
+                        v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (has_cols && j0 + j < n)
+                            v[j] = *reinterpret_cast<const float4*>(a.part_o + (size_t)row * HD + 4 * lane);
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < kPartBatch; ++j) {
+                    const float w = __shfl_sync(0xffffffffu, my_w, (j0 + j) & 31);   // 0 past the end of the list
+                    const float wj = (j0 + j < n) ? w : 0.f;
+                    acc.x += wj * v[j].x;
+                    acc.y += wj * v[j].y;
+                    acc.z += wj * v[j].z;
+                    acc.w += wj * v[j].w;
+                }
             }
         }
     }
     if (has_cols) *reinterpret_cast<float4*>(a.out + (size_t)bh * HD + 4 * lane) = acc;   // zeros when there are no parts
 
-    if (a.block_mass != nullptr && hi > lo) {
-        const int nblk = a.plan.br_nblk[b];
-        float* mass = a.block_mass + a.plan.mass_off[b] * a.Hq + (int64_t)h * nblk;
-        const int stride = 32 * wpk;
-        int j = sub * 32 + lane;
-        for (; j + 3 * stride < nblk; j += 4 * stride) {   // four independent loads in flight
-            const float v0 = mass[j], v1 = mass[j + stride], v2 = mass[j + 2 * stride], v3 = mass[j + 3 * stride];
-            mass[j] = fast_exp2(v0 - lse);
-            mass[j + stride] = fast_exp2(v1 - lse);
-            mass[j + 2 * stride] = fast_exp2(v2 - lse);
-            mass[j + 3 * stride] = fast_exp2(v3 - lse);
+    // block masses: mass_j = 2^(logmass_j - LSE), in place
+    for (int j0 = sub * 32 + lane; j0 < nblk; j0 += kMassBatch * stride) {
+        if (j0 != sub * 32 + lane) {
+#pragma unroll
+            for (int k = 0; k < kMassBatch; ++k) {
+                const int j = j0 + k * stride;
+                mv[k] = (j < nblk) ? mass[j] : 0.f;
+            }
         }
-        for (; j < nblk; j += stride) mass[j] = fast_exp2(mass[j] - lse);
+#pragma unroll
+        for (int k = 0; k < kMassBatch; ++k) {
+            const int j = j0 + k * stride;
+            if (j < nblk) mass[j] = fast_exp2(mv[k] - lse);
+        }
     }
 }
 
