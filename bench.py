@@ -64,6 +64,8 @@ def parse_args():
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-config attention-only table")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-pipeline", action="store_true", help="time the steps strictly one after another")
+    ap.add_argument("--pipeline-depth", type=int, default=4,
+                    help="steps in flight in the headline loop (streams and buffer sets); depth - 2 host threads build plans")
     ap.add_argument("--cgee-only", action="store_true",
                     help="run only the CGEE entropy-kernel measurement and print its object (used for profiling)")
     ap.add_argument("--model-step-only", action="store_true",
@@ -214,13 +216,19 @@ def run_step(rk, batch: DeviceBatch, seg_events=None):
 
 
 class StepContext:
-    """Per-step buffers and stream for the software-pipelined loop (two steps in flight)."""
+    """Per-step buffers for the software-pipelined loop.  All contexts share two streams: one for the gate
+    kernels and their map copies, one for the attention calls, so that attention launches run back to back
+    in step order (two persistent attention kernels at once only take SMs from each other) while the gates
+    of later steps slip in beside them."""
+    streams = None
 
     def __init__(self, batch: DeviceBatch, plan):
         import torch
         dev = batch.dev
         B = batch.q.shape[0]
-        self.stream = torch.cuda.Stream(device=dev)
+        if StepContext.streams is None:
+            StepContext.streams = (torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev))
+        self.gate_stream, self.stream = StepContext.streams
         self.map_dev = torch.empty(B, dtype=torch.int32, device=dev)
         self.sigma_dev = torch.empty(B, dtype=torch.float32, device=dev)
         self.map_host = torch.empty(B, dtype=torch.int32).pin_memory()
@@ -233,9 +241,10 @@ class StepContext:
 
 
 def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events, pool):
-    """K steps, software-pipelined three deep over len(ctxs) = 3 contexts (stream + buffers each):
-    while the attention of step i runs, the gate kernel of step i+2 is already enqueued and a host
-    worker thread builds step i+1's plan from its map (the C calls release the interpreter lock).
+    """K steps, software-pipelined over n = len(ctxs) contexts (stream + buffers each): while the
+    attention of step i runs, the gate kernels of the next n - 1 steps are already enqueued and host
+    worker threads build the plans of the next n - 2 steps from their maps (the C calls release the
+    interpreter lock).
     Every step still does the whole path: gate kernel, map to the host, tables + plan, segment
     kernels, merge.  Returns the number of kernel launches."""
     import torch
@@ -247,10 +256,10 @@ def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events, pool):
     def gate_stage(ctx):
         launches[0] += 1
         rk.rksc_asks_gate(batch.h_branch, batch.h_root, batch.cand, g.alpha, g.tau,
-                          branch_to_prefix=ctx.map_dev, sigma=ctx.sigma_dev, stream=ctx.stream)
-        with torch.cuda.stream(ctx.stream):
+                          branch_to_prefix=ctx.map_dev, sigma=ctx.sigma_dev, stream=ctx.gate_stream)
+        with torch.cuda.stream(ctx.gate_stream):
             ctx.map_host.copy_(ctx.map_dev, non_blocking=True)
-        ctx.ev_map.record(ctx.stream)
+        ctx.ev_map.record(ctx.gate_stream)
 
     def plan_stage(ctx):
         ctx.ev_map.synchronize()                       # the host needs the map to build the tables
@@ -269,16 +278,20 @@ def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events, pool):
         launches[0] += plan.num_kernel_launches
         ctx.plan = plan                                # the context's previous plan is released here
 
-    gate_stage(ctxs[0])
-    if steps > 1:
-        gate_stage(ctxs[1 % n])
-    fut = pool.submit(plan_stage, ctxs[0])
+    # gates run n - 1 steps ahead of the attention, plans n - 2 (one worker thread each)
+    from collections import deque
+    ahead_gate, ahead_plan = n - 1, max(1, n - 2)
+    futs = deque()
+    for i in range(min(ahead_gate, steps)):
+        gate_stage(ctxs[i % n])
+    for i in range(min(ahead_plan, steps)):
+        futs.append(pool.submit(plan_stage, ctxs[i % n]))
     for i in range(steps):
-        if i + 2 < steps:
-            gate_stage(ctxs[(i + 2) % n])
-        nxt = pool.submit(plan_stage, ctxs[(i + 1) % n]) if i + 1 < steps else None
-        attention_stage(ctxs[i % n], fut.result(), seg_events.get(i))
-        fut = nxt
+        if i + ahead_gate < steps:
+            gate_stage(ctxs[(i + ahead_gate) % n])
+        if i + ahead_plan < steps:
+            futs.append(pool.submit(plan_stage, ctxs[(i + ahead_plan) % n]))
+        attention_stage(ctxs[i % n], futs.popleft().result(), seg_events.get(i))
     return launches[0]
 
 
@@ -455,8 +468,9 @@ def run_ours(args):
     if pipelined:
         # the headline loop: two steps in flight on two streams (see pipelined_steps)
         from concurrent.futures import ThreadPoolExecutor
-        pool = ThreadPoolExecutor(max_workers=1)
-        ctxs = [StepContext(batch, plan) for _ in range(3)]
+        depth = max(3, args.pipeline_depth)
+        pool = ThreadPoolExecutor(max_workers=depth - 2)
+        ctxs = [StepContext(batch, plan) for _ in range(depth)]
         pipelined_steps(rk, batch, ctxs, 6, {}, pool)
         torch.cuda.synchronize()
         # events around the segment kernels on every 4th step (they cost two extra host calls)
@@ -466,11 +480,11 @@ def run_ours(args):
         barrier()
         t_wall0 = time.perf_counter()
         e_start.record()
-        for c in ctxs:
-            c.stream.wait_event(e_start)
+        for st in StepContext.streams:
+            st.wait_event(e_start)
         launches = pipelined_steps(rk, batch, ctxs, args.steps, seg_ev, pool)
-        for c in ctxs:
-            torch.cuda.current_stream().wait_stream(c.stream)
+        for st in StepContext.streams:
+            torch.cuda.current_stream().wait_stream(st)
         e_end.record()
         barrier()
         t_wall = time.perf_counter() - t_wall0
@@ -493,8 +507,9 @@ def run_ours(args):
         "config": {
             "workload": WORKLOAD_LABEL[args.workload],
             "step": "gate kernel + map D2H + tables + plan + attention (segment kernels + merge)",
-            "pipelining": ("three steps in flight (3 streams): while the attention of step i runs, the gate of step "
-                           "i+2 is enqueued and a host thread builds the plan of step i+1") if pipelined
+            "pipelining": (f"{depth} steps in flight ({depth} streams): while the attention of step i runs, the gates of "
+                           f"steps i+1..i+{depth - 1} are enqueued and {depth - 2} host threads build the plans of steps "
+                           f"i+1..i+{depth - 2}") if pipelined
             else "none (steps strictly serial)",
             "unique_kv_bytes": kv_bytes, "branches": B, "work_items": plan.num_work_items,
             "l2": ("inputs larger than L2 (unique KV %.0f MB vs L2 %.0f MB)" % (kv_bytes / 1e6, l2_bytes / 1e6))

@@ -443,12 +443,39 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
 
 namespace {
 
+// The per-step device buffers come from a memory pool of the library's own, one per device, that
+// keeps what is freed: the device's default pool hands freed memory back to the system at every
+// synchronisation (release threshold 0), and mapping a hundred megabytes anew each step costs
+// milliseconds.  The pool holds about one step's buffers between calls.
+cudaMemPool_t g_step_pool[kMaxDevices];
+bool g_step_pool_ready[kMaxDevices];
+
+cudaError_t step_pool(int dev, cudaMemPool_t* pool) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_step_pool_ready[dev]) {
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        cudaError_t e = cudaMemPoolCreate(&g_step_pool[dev], &props);
+        if (e != cudaSuccess) return e;
+        uint64_t keep = UINT64_MAX;
+        e = cudaMemPoolSetAttribute(g_step_pool[dev], cudaMemPoolAttrReleaseThreshold, &keep);
+        if (e != cudaSuccess) return e;
+        g_step_pool_ready[dev] = true;
+    }
+    *pool = g_step_pool[dev];
+    return cudaSuccess;
+}
+
 struct AsyncBuf {   // stream-ordered device buffer, released on scope exit
     void* p = nullptr;
     cudaStream_t s = nullptr;
+    cudaMemPool_t pool = nullptr;
     cudaError_t alloc(size_t bytes, cudaStream_t stream) {
         s = stream;
-        return cudaMallocAsync(&p, bytes ? bytes : 16, stream);
+        return cudaMallocFromPoolAsync(&p, bytes ? bytes : 16, pool, stream);
     }
     ~AsyncBuf() {
         if (p) cudaFreeAsync(p, s);
@@ -467,13 +494,20 @@ extern "C" RKSC_API int32_t rksc_decode_step_host(
     if (!layout || !h_branch || !h_root || !cand_prefix || !q || !k_pool || !v_pool || !branch_to_prefix || !out)
         return RKSC_ERR_INVALID_ARG;
     if (B <= 0 || P <= 0 || L <= 0 || D <= 0) return RKSC_ERR_INVALID_ARG;
-    int32_t st = ensure_device(nullptr);
+    int dev = -1;
+    int32_t st = ensure_device(&dev);
     if (st != RKSC_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaMemPool_t pool = nullptr;
+    if (step_pool(dev, &pool) != cudaSuccess) {
+        g_last_cuda = cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
     const size_t nb = (size_t)B * L * D * sizeof(float), nr = (size_t)P * L * D * sizeof(float);
     const size_t nq = (size_t)B * layout->num_q_heads * layout->head_dim * 2;
     const size_t nout = (size_t)B * layout->num_q_heads * layout->head_dim * sizeof(float);
     AsyncBuf d_hb, d_hr, d_cand, d_map, d_sigma, d_q, d_out, d_mass, d_ws, d_status;
+    for (AsyncBuf* b : {&d_hb, &d_hr, &d_cand, &d_map, &d_sigma, &d_q, &d_out, &d_mass, &d_ws, &d_status}) b->pool = pool;
     cudaError_t e = cudaSuccess;
     auto ok = [&](cudaError_t r) {
         if (e == cudaSuccess && r != cudaSuccess) e = r;

@@ -65,6 +65,15 @@ __device__ __forceinline__ void cg_tma_2d(uint32_t dst, const CUtensorMap* tm, i
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+// W_u is read once per call: its lines are the first to leave L2 again.
+__device__ __forceinline__ void cg_tma_2d_stream(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar), "l"(policy)
+        : "memory");
+}
 __device__ __forceinline__ void cg_ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -145,6 +154,8 @@ logit_entropy_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         if (lane == 0) {
             cg_mbar_expect_tx(bars + 8 * 2 * kCgStages, (uint32_t)nkc * (uint32_t)kHChunk);
             for (int kc = 0; kc < nkc; ++kc) cg_tma_2d(hbase + kc * kHChunk, &tm_h, kc * 64, 0, bars + 8 * 2 * kCgStages);
+            uint64_t w_policy;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(w_policy));
             uint32_t seq = 0;
             for (long long tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x) {
                 for (int kc = 0; kc < nkc && !*abort_flag; ++kc, ++seq) {
@@ -152,7 +163,7 @@ logit_entropy_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
                     if (seq >= kCgStages) wait_or_abort(bars + 8 * (kCgStages + st), (seq / kCgStages - 1) & 1u);
                     if (*abort_flag) break;
                     cg_mbar_expect_tx(bars + 8 * st, kCgStageBytes);
-                    cg_tma_2d(ring + st * kCgStageBytes, &tm_w, kc * 64, (int)(tile * kCgTileRows), bars + 8 * st);
+                    cg_tma_2d_stream(ring + st * kCgStageBytes, &tm_w, kc * 64, (int)(tile * kCgTileRows), bars + 8 * st, w_policy);
                 }
             }
         }
