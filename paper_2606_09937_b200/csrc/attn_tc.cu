@@ -317,8 +317,6 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         mbar_init(bar(kBarEpiB), kSmWarps);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // the kernels that follow on the stream may be made resident early; they wait themselves
-        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     }
     if (warp == kMmaWarp) {   // one warp allocates (and later frees) the tensor memory
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + kTmemPtrOff),
@@ -330,6 +328,13 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *s_tmem;
+    // Launched with programmatic stream serialisation: everything above (barriers, tensor memory) may
+    // run while the kernel before this one on the stream is still draining; nothing below, which reads
+    // what that kernel may have written (queries, pool, claim counters) and writes what it may still
+    // read (partial results, masses), starts before it has completed.  Only then may the kernels after
+    // this one be made resident: the warp-MMA kernel does not wait at its start.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     auto wait_or_abort = [&](uint32_t b, uint32_t parity) {
         if (*s_abort) return;
@@ -861,8 +866,17 @@ cudaError_t configure_tc_kernel() {
 cudaError_t launch_seg_attn_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnArgs& a,
                                cudaStream_t stream) {
     if (a.grid_tc == 0) return cudaSuccess;
-    seg_attn_tc_kernel<<<a.grid_tc, kTcThreads, tc_kernel_smem_bytes(), stream>>>(tm_k, tm_v, a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.grid_tc, 1, 1);
+    cfg.blockDim = dim3(kTcThreads, 1, 1);
+    cfg.dynamicSmemBytes = tc_kernel_smem_bytes();
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, seg_attn_tc_kernel, tm_k, tm_v, a);
 }
 
 }  // namespace rksc

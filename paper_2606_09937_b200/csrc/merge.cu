@@ -57,6 +57,9 @@ merge_kernel(const AttnArgs a, const int wpk_log2) {
     // the first 32 part rows of this warp's list (plan data: readable before the dependency resolves)
     const int row_l = (lo + lane < hi) ? a.plan.merge_rows[lo + lane] + gi : -1;
 
+    // a kernel launched behind this one with programmatic serialisation may set itself up meanwhile
+    // (it waits for this grid's completion before it touches memory)
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // everything below reads what the segment kernel wrote
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (!live) return;
