@@ -471,7 +471,8 @@ def run_ours(args):
         depth = max(3, args.pipeline_depth)
         pool = ThreadPoolExecutor(max_workers=depth - 2)
         ctxs = [StepContext(batch, plan) for _ in range(depth)]
-        pipelined_steps(rk, batch, ctxs, 6, {}, pool)
+        # untimed: the requested warm-up steps, and enough more that both host threads and all buffer sets have run
+        pipelined_steps(rk, batch, ctxs, max(args.warmup, 3) + 4 * depth, {}, pool)
         torch.cuda.synchronize()
         # events around the segment kernels on every 4th step (they cost two extra host calls)
         seg_ev = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
