@@ -693,23 +693,20 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 float mx = -INFINITY;
                 if (warp_has_rows) {
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
+                    // the maximum is taken over the raw scores (the scale is positive) and scaled once; the
+                    // scale itself is applied inside the exponent's multiply-add below
                     if (nvalid >= kSlotTokens) {
 #pragma unroll
-                        for (int j = 0; j < 64; ++j) {
-                            const float v = __uint_as_float(sr[j >> 5][j & 31]) * scale_log2;
-                            sr[j >> 5][j & 31] = __float_as_uint(v);
-                            mx4[j & 3] = fmaxf(mx4[j & 3], v);
-                        }
+                        for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sr[j >> 5][j & 31]));
                     } else {
 #pragma unroll
                         for (int j = 0; j < 64; ++j) {
-                            float v = __uint_as_float(sr[j >> 5][j & 31]) * scale_log2;
-                            v = (j < nvalid) ? v : -INFINITY;
+                            const float v = (j < nvalid) ? __uint_as_float(sr[j >> 5][j & 31]) : -INFINITY;
                             sr[j >> 5][j & 31] = __float_as_uint(v);
                             mx4[j & 3] = fmaxf(mx4[j & 3], v);
                         }
                     }
-                    mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                    mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
                 }
 
                 // Running maximum with slack: m is raised (and O, l rescaled) only when a row's maximum
@@ -741,7 +738,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 }
 
                 // p = 2^(s - m), its per-page sums, and the P row as bf16 pairs (A operand of P V) in two
-                // parts: the upper 16 bits of p, and the rest rounded to bf16.  One bf16 alone carries
+                // parts: the upper 16 bits of p, and the upper 16 bits of the rest.  One bf16 alone carries
                 // 2^-9 relative error into the output, more than its tolerance when few tokens hold most of
                 // a row's mass; P V is accumulated over both parts.
                 float ps[4] = {0.f, 0.f, 0.f, 0.f};
@@ -750,14 +747,14 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     const float mm = valid ? m : 0.f;   // rows past the item's end: harmless, never read
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        const float p0 = fast_exp2(__uint_as_float(sr[(2 * j) >> 5][(2 * j) & 31]) - mm);
-                        const float p1 = fast_exp2(__uint_as_float(sr[(2 * j + 1) >> 5][(2 * j + 1) & 31]) - mm);
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[(2 * j) >> 5][(2 * j) & 31]), scale_log2, -mm));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[(2 * j + 1) >> 5][(2 * j + 1) & 31]), scale_log2, -mm));
                         ps[j >> 3] += p0;
                         ps[j >> 3] += p1;
                         const uint32_t h0 = __float_as_uint(p0) & 0xffff0000u, h1 = __float_as_uint(p1) & 0xffff0000u;
                         pk[j] = __byte_perm(h0, h1, 0x7632);   // (h1 upper half, h0 upper half)
-                        const __nv_bfloat162 lo2 = __floats2bfloat162_rn(p0 - __uint_as_float(h0), p1 - __uint_as_float(h1));
-                        pl[j] = *reinterpret_cast<const uint32_t*>(&lo2);
+                        // the rest, p - upper part (exact in fp32), cut to its own upper 16 bits: 2^-16 of p is lost
+                        pl[j] = __byte_perm(__float_as_uint(p0 - __uint_as_float(h0)), __float_as_uint(p1 - __uint_as_float(h1)), 0x7632);
                     }
                 } else {
 #pragma unroll
