@@ -402,6 +402,55 @@ RKSC_API int32_t rksc_tables_append_token(const rksc_tables* in, const int32_t* 
 RKSC_API int32_t rksc_kv_append(const rksc_layout* layout, void* k_pool, void* v_pool, const void* k_new,
                                 const void* v_new, int32_t B, const int32_t* page, const int32_t* slot, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Step pipeline: whole steps of the path (gate -> map to the host -> tables + plan -> attention,
+ * paper Algorithm 1 lines 2-4 restricted to ASKS and the decode attention) kept `depth` deep in
+ * flight by the library itself, for callers whose steps do not depend on each other's results
+ * (independent batches, the layers' gates of later requests, a serving loop).
+ *
+ * The tables of a step depend on its gate map, which has to come to the host; a caller that runs
+ * the four stages one after another leaves the GPU idle while the host builds the plan.  The
+ * pipeline owns two streams and depth - 2 (at least one) host threads: rksc_pipeline_submit
+ * enqueues the step's gate kernel and the copy of its map on the gate stream and returns; a host
+ * thread waits for that copy, builds tables and plan, and enqueues the attention on the attention
+ * stream - in submission order, so that attention launches run back to back while the gates of
+ * later steps run beside them.
+ *
+ * rksc_pipeline_create: layout, shapes (B branches, P prefixes, L layers, D hidden size), alpha,
+ *   tau and the three page-list CSRs as for rksc_tables_from_gate (host arrays, copied: every step
+ *   uses the same lists, only its gate map differs); depth in [2, 8]; mass_capacity = floats the
+ *   caller's block_mass buffers hold (0 if it passes none); timing != 0 makes every step record
+ *   CUDA events around its segment kernels (the attention is then launched in its two phases).
+ * rksc_pipeline_submit: device pointers as for rksc_asks_gate (h_branch, h_root, cand_prefix) and
+ *   rksc_branch_decode_attention (q, pools, out, block_mass or NULL).  The buffers must stay valid
+ *   and unchanged until the step has been waited for; `after_stream` (may be NULL): work already
+ *   enqueued on that stream is waited for by the step (its inputs' producers).  Never blocks; at
+ *   most `depth` steps may be in flight: RKSC_ERR_INVALID_ARG if step ticket - depth has not been
+ *   waited for yet.  *ticket identifies the step (0, 1, 2, ...).  The calling thread's current
+ *   device must be the one the pipeline was created on.
+ * rksc_pipeline_wait: blocks the calling thread until step `ticket` has finished; tickets must be
+ *   waited for in submission order, each once.  Optional outputs (host, may be NULL):
+ *   branch_to_prefix [B], sigma [B], mass_off [B+1], info (the step's plan), segment_ms (timing
+ *   pipelines: device time of the step's segment kernels).  Returns the first failing stage's status, or
+ *   the attention's device status word, or RKSC_ERR_WORKSPACE when the step's masses did not fit
+ *   mass_capacity (the attention was not run).
+ * rksc_pipeline_destroy: waits for everything in flight, stops the threads, frees the buffers.
+ * Thread safety: one submitting / waiting thread per pipeline.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct rksc_pipeline rksc_pipeline;
+RKSC_API int32_t rksc_pipeline_create(const rksc_layout* layout, int32_t B, int32_t P, int32_t L, int32_t D,
+                                      float alpha, float tau,
+                                      const int32_t* shared_off, const int32_t* shared_pages, const int32_t* shared_ntok,
+                                      const int32_t* priv_off, const int32_t* priv_pages, const int32_t* priv_ntok,
+                                      const int32_t* sfx_off, const int32_t* sfx_pages, const int32_t* sfx_ntok,
+                                      int32_t depth, int64_t mass_capacity, int32_t timing, rksc_pipeline** out);
+RKSC_API int32_t rksc_pipeline_submit(rksc_pipeline* pipe, const float* h_branch, const float* h_root,
+                                      const int32_t* cand_prefix, const void* q, const void* k_pool, const void* v_pool,
+                                      float* out, float* block_mass, void* after_stream, int64_t* ticket);
+RKSC_API int32_t rksc_pipeline_wait(rksc_pipeline* pipe, int64_t ticket, int32_t* branch_to_prefix, float* sigma,
+                                    int64_t* mass_off, rksc_plan_info* info, float* segment_ms);
+RKSC_API void    rksc_pipeline_destroy(rksc_pipeline* pipe);
+
 #ifdef __cplusplus
 }
 #endif

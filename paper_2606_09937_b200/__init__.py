@@ -32,6 +32,8 @@ from .binding import (  # noqa: F401
     rksc_cgee_logit_entropy,
     rksc_cgee_entropy_exit,
     rksc_cgee_verify_skip,
+    Pipeline,
+    StepResult,
     STATIC_WORKSPACE_BYTES,
     split_block_mass,
     EXPORTED_SYMBOLS,

@@ -42,6 +42,10 @@ EXPORTED_SYMBOLS = (
     "rksc_cgee_logit_entropy",
     "rksc_cgee_entropy_exit",
     "rksc_cgee_verify_skip",
+    "rksc_pipeline_create",
+    "rksc_pipeline_submit",
+    "rksc_pipeline_wait",
+    "rksc_pipeline_destroy",
 )
 STATIC_WORKSPACE_BYTES = 16 << 20
 
@@ -147,6 +151,16 @@ def lib() -> C.CDLL:
     L.rksc_tables_for_suffix_prefill.argtypes = [C.POINTER(_CTables), C.c_int32, C.POINTER(_CTables)]
     L.rksc_tables_drop_evicted.restype = C.c_int32
     L.rksc_tables_drop_evicted.argtypes = [C.POINTER(_CTables), C.c_void_p, C.POINTER(_CTables)]
+    L.rksc_pipeline_create.restype = C.c_int32
+    L.rksc_pipeline_create.argtypes = ([C.POINTER(_CLayout)] + [C.c_int32] * 4 + [C.c_float, C.c_float] + [i32p] * 9 +
+                                       [C.c_int32, C.c_int64, C.c_int32, C.POINTER(C.c_void_p)])
+    L.rksc_pipeline_submit.restype = C.c_int32
+    L.rksc_pipeline_submit.argtypes = [C.c_void_p] * 10 + [C.POINTER(C.c_int64)]
+    L.rksc_pipeline_wait.restype = C.c_int32
+    L.rksc_pipeline_wait.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(_CPlanInfo),
+                                     C.POINTER(C.c_float)]
+    L.rksc_pipeline_destroy.restype = None
+    L.rksc_pipeline_destroy.argtypes = [C.c_void_p]
     _lib = L
     return L
 
@@ -585,3 +599,73 @@ def rksc_decode_step_host(layout, h_branch, h_root, cand_prefix, alpha, tau, fla
         block_mass.numel() if block_mass is not None else 0, mo, _stream_ptr(stream, k_pool.device))
     _check(st, "rksc_decode_step_host")
     return st
+
+
+class StepResult:
+    """What rksc_pipeline_wait hands back for one step (host data)."""
+
+    def __init__(self, status, branch_to_prefix, sigma, mass_off, info, segment_ms):
+        self.status = status
+        self.branch_to_prefix = branch_to_prefix
+        self.sigma = sigma
+        self.mass_off = mass_off
+        self.mass_elems = int(info.mass_elems)
+        self.workspace_bytes = int(info.workspace_bytes)
+        self.num_work_items = int(info.num_work_items)
+        self.num_kernel_launches = int(info.num_kernel_launches)
+        self.unique_kv_tokens = int(info.unique_kv_tokens)
+        self.num_pages_listed = int(info.num_pages_listed)
+        self.segment_ms = segment_ms
+
+
+class Pipeline:
+    """rksc_pipeline_*: whole steps (gate, map to the host, tables + plan, attention) kept ``depth`` deep in
+    flight by the library's own streams and host threads.  Argument marshalling only."""
+
+    def __init__(self, layout, num_branches, hidden_shape, alpha, tau, lists, depth=4, mass_capacity=0, timing=False):
+        lay = layout if isinstance(layout, Layout) else Layout.of(layout)
+        gl = lists if isinstance(lists, GateLists) else GateLists(lists)
+        L_, D = hidden_shape
+        self.layout, self.B, self.depth = lay, int(num_branches), int(depth)
+        h = C.c_void_p()
+        _check(lib().rksc_pipeline_create(C.byref(lay.c), self.B, gl.num_prefixes, int(L_), int(D), float(alpha),
+                                          float(tau), *gl.ptrs, int(depth), int(mass_capacity), int(bool(timing)),
+                                          C.byref(h)), "rksc_pipeline_create")
+        self._h = h.value
+        self._keep = {}
+
+    def submit(self, h_branch, h_root, cand_prefix, q, k_pool, v_pool, out, block_mass=None, after_stream=None) -> int:
+        t = C.c_int64(-1)
+        _check(lib().rksc_pipeline_submit(self._h, h_branch.data_ptr(), h_root.data_ptr(), cand_prefix.data_ptr(),
+                                          q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), out.data_ptr(),
+                                          block_mass.data_ptr() if block_mass is not None else None,
+                                          _stream_ptr(after_stream, q.device) if after_stream is not None else None,
+                                          C.byref(t)), "rksc_pipeline_submit")
+        # the step reads these buffers until it has been waited for
+        self._keep[t.value] = (h_branch, h_root, cand_prefix, q, k_pool, v_pool, out, block_mass)
+        return int(t.value)
+
+    def wait(self, ticket: int, check: bool = True) -> StepResult:
+        m = np.empty(self.B, dtype=np.int32)
+        sg = np.empty(self.B, dtype=np.float32)
+        mo = np.zeros(self.B + 1, dtype=np.int64)
+        info = _CPlanInfo()
+        ms = C.c_float(0.0)
+        st = lib().rksc_pipeline_wait(self._h, int(ticket), m.ctypes.data, sg.ctypes.data, mo.ctypes.data,
+                                      C.byref(info), C.byref(ms))
+        self._keep.pop(int(ticket), None)
+        if check:
+            _check(st, "rksc_pipeline_wait")
+        return StepResult(int(st), m, sg, mo, info, float(ms.value))
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().rksc_pipeline_destroy(self._h)
+            self._h = None
+            self._keep.clear()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 REPO_DIR = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "librksc.so")
-SOURCES = ["api.cu", "plan.cpp", "gate.cu", "attn_warp.cu", "attn_tc.cu", "merge.cu", "rsbcm.cu", "cgee.cu"]
+SOURCES = ["api.cu", "plan.cpp", "gate.cu", "attn_warp.cu", "attn_tc.cu", "merge.cu", "rsbcm.cu", "cgee.cu", "pipeline.cpp"]
 HEADERS = ["rksc_internal.h", "kernels.h"]
 
 
