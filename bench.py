@@ -65,7 +65,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-pipeline", action="store_true", help="time the steps strictly one after another")
     ap.add_argument("--pipeline-depth", type=int, default=4,
-                    help="steps in flight in the headline loop (streams and buffer sets); depth - 2 host threads build plans")
+                    help="steps the library's pipeline keeps in flight in the headline loop (2..8; depth - 2 host threads)")
     ap.add_argument("--cgee-only", action="store_true",
                     help="run only the CGEE entropy-kernel measurement and print its object (used for profiling)")
     ap.add_argument("--model-step-only", action="store_true",
@@ -213,86 +213,6 @@ def run_step(rk, batch: DeviceBatch, seg_events=None):
         rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=2, **kw)
     launches += plan.num_kernel_launches
     return plan, launches
-
-
-class StepContext:
-    """Per-step buffers for the software-pipelined loop.  All contexts share two streams: one for the gate
-    kernels and their map copies, one for the attention calls, so that attention launches run back to back
-    in step order (two persistent attention kernels at once only take SMs from each other) while the gates
-    of later steps slip in beside them."""
-    streams = None
-
-    def __init__(self, batch: DeviceBatch, plan):
-        import torch
-        dev = batch.dev
-        B = batch.q.shape[0]
-        if StepContext.streams is None:
-            StepContext.streams = (torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev))
-        self.gate_stream, self.stream = StepContext.streams
-        self.map_dev = torch.empty(B, dtype=torch.int32, device=dev)
-        self.sigma_dev = torch.empty(B, dtype=torch.float32, device=dev)
-        self.map_host = torch.empty(B, dtype=torch.int32).pin_memory()
-        self.ev_map = torch.cuda.Event()
-        self.out = torch.empty_like(batch.out)
-        self.mass = torch.empty_like(batch.mass)
-        self.workspace = torch.empty_like(batch.workspace)
-        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.plan = None
-
-
-def pipelined_steps(rk, batch: DeviceBatch, ctxs, steps: int, seg_events, pool):
-    """K steps, software-pipelined over n = len(ctxs) contexts (stream + buffers each): while the
-    attention of step i runs, the gate kernels of the next n - 1 steps are already enqueued and host
-    worker threads build the plans of the next n - 2 steps from their maps (the C calls release the
-    interpreter lock).
-    Every step still does the whole path: gate kernel, map to the host, tables + plan, segment
-    kernels, merge.  Returns the number of kernel launches."""
-    import torch
-    w = batch.w
-    g = w.gate
-    n = len(ctxs)
-    launches = [0]
-
-    def gate_stage(ctx):
-        launches[0] += 1
-        rk.rksc_asks_gate(batch.h_branch, batch.h_root, batch.cand, g.alpha, g.tau,
-                          branch_to_prefix=ctx.map_dev, sigma=ctx.sigma_dev, stream=ctx.gate_stream)
-        with torch.cuda.stream(ctx.gate_stream):
-            ctx.map_host.copy_(ctx.map_dev, non_blocking=True)
-        ctx.ev_map.record(ctx.gate_stream)
-
-    def plan_stage(ctx):
-        ctx.ev_map.synchronize()                       # the host needs the map to build the tables
-        return rk.rksc_plan_create_from_gate(batch.layout, ctx.map_host.numpy(), batch.lists)
-
-    def attention_stage(ctx, plan, ev):
-        kw = dict(out=ctx.out, block_mass=ctx.mass, workspace=ctx.workspace, device_status=ctx.status,
-                  stream=ctx.stream)
-        if ev is None:
-            rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, **kw)
-        else:                                          # every few steps: events around the segment kernels
-            ev[0].record(ctx.stream)
-            rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=1, **kw)
-            ev[1].record(ctx.stream)
-            rk.rksc_branch_decode_attention(plan, batch.q, batch.k_pool, batch.v_pool, phases=2, **kw)
-        launches[0] += plan.num_kernel_launches
-        ctx.plan = plan                                # the context's previous plan is released here
-
-    # gates run n - 1 steps ahead of the attention, plans n - 2 (one worker thread each)
-    from collections import deque
-    ahead_gate, ahead_plan = n - 1, max(1, n - 2)
-    futs = deque()
-    for i in range(min(ahead_gate, steps)):
-        gate_stage(ctxs[i % n])
-    for i in range(min(ahead_plan, steps)):
-        futs.append(pool.submit(plan_stage, ctxs[i % n]))
-    for i in range(steps):
-        if i + ahead_gate < steps:
-            gate_stage(ctxs[(i + ahead_gate) % n])
-        if i + ahead_plan < steps:
-            futs.append(pool.submit(plan_stage, ctxs[(i + ahead_plan) % n]))
-        attention_stage(ctxs[i % n], futs.popleft().result(), seg_events.get(i))
-    return launches[0]
 
 
 def attention_only_times(rk, batch: DeviceBatch, plan, iters: int, flush):
@@ -466,34 +386,55 @@ def run_ours(args):
               "what": "the same K steps strictly one after another on one stream"}
     pipelined = batch.has_gate and not small and not args.no_pipeline
     if pipelined:
-        # the headline loop: two steps in flight on two streams (see pipelined_steps)
-        from concurrent.futures import ThreadPoolExecutor
-        depth = max(3, args.pipeline_depth)
-        pool = ThreadPoolExecutor(max_workers=depth - 2)
-        ctxs = [StepContext(batch, plan) for _ in range(depth)]
-        # untimed: the requested warm-up steps, and enough more that both host threads and all buffer sets have run
-        pipelined_steps(rk, batch, ctxs, max(args.warmup, 3) + 4 * depth, {}, pool)
+        # the headline loop: the library's step pipeline (rksc_pipeline_*) keeps `depth` whole steps in flight on
+        # its own gate stream, attention stream and host threads; this thread only submits and waits
+        depth = max(2, min(8, args.pipeline_depth))
+        g, f = w.gate, w.flat
+        B = w.num_branches
+        cap = 0
+        for b in range(B):
+            r = int(g.cand_prefix[b])
+            cap += max(int(f.shared_off[r + 1] - f.shared_off[r]), int(f.priv_off[b + 1] - f.priv_off[b]))
+            cap += int(f.sfx_off[b + 1] - f.sfx_off[b])
+        cap *= w.layout.num_q_heads                      # block masses of a step whatever its gate map
+        pipe = rk.Pipeline(batch.layout, B, tuple(g.h_branch.shape[1:]), g.alpha, g.tau, batch.lists, depth=depth,
+                           mass_capacity=cap, timing=True)
+        bufs = [(torch.empty_like(batch.out), torch.empty(cap, dtype=torch.float32, device=dev)) for _ in range(depth)]
+        ticket = [0]
+
+        def run_pipeline(nsteps, after=None):
+            """Submits nsteps steps, never more than `depth` in flight; returns their results."""
+            res, first = [], ticket[0]
+            for i in range(nsteps):
+                t = ticket[0]
+                if t - first >= depth:
+                    res.append(pipe.wait(t - depth))
+                o, m = bufs[t % depth]
+                pipe.submit(batch.h_branch, batch.h_root, batch.cand, batch.q, batch.k_pool, batch.v_pool, o, m,
+                            after_stream=after if i == 0 else None)
+                ticket[0] = t + 1
+            for t in range(max(first, ticket[0] - depth), ticket[0]):
+                res.append(pipe.wait(t))
+            return res
+
+        run_pipeline(max(args.warmup, 3) + 2 * depth)         # untimed warm-up
         torch.cuda.synchronize()
-        # events around the segment kernels on every 4th step (they cost two extra host calls)
-        seg_ev = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                  for i in range(0, args.steps, 4)}
         e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         t_wall0 = time.perf_counter()
         e_start.record()
-        for st in StepContext.streams:
-            st.wait_event(e_start)
-        launches = pipelined_steps(rk, batch, ctxs, args.steps, seg_ev, pool)
-        for st in StepContext.streams:
-            torch.cuda.current_stream().wait_stream(st)
+        # the first step waits for e_start through `after`; the last wait returns when the last step has finished
+        results = run_pipeline(args.steps, after=torch.cuda.current_stream())
         e_end.record()
         barrier()
         t_wall = time.perf_counter() - t_wall0
-        pool.shutdown()
         total_ms = e_start.elapsed_time(e_end)
-        seg_ms = [a.elapsed_time(b) for a, b in seg_ev.values()]
-        for c in ctxs:
-            assert int(c.status.item()) == 0, "a kernel reported a device-side timeout"
+        assert len(results) == args.steps and all(r.status == 0 for r in results)
+        seg_ms = [r.segment_ms for r in results]
+        launches = sum(1 + r.num_kernel_launches for r in results)
+        assert all(np.array_equal(r.branch_to_prefix, batch.map_host.numpy()) for r in results[:3])
+        pipe.close()
+        del bufs
     clocks = sampler.stop() if rank == 0 else None
     value, total_ms_max = aggregate_over_ranks(dist, dev, kv_bytes, args.steps, total_ms)
     peak_gbs, peak_kind = measured_peak_gbs()
@@ -508,9 +449,10 @@ def run_ours(args):
         "config": {
             "workload": WORKLOAD_LABEL[args.workload],
             "step": "gate kernel + map D2H + tables + plan + attention (segment kernels + merge)",
-            "pipelining": (f"{depth} steps in flight ({depth} streams): while the attention of step i runs, the gates of "
-                           f"steps i+1..i+{depth - 1} are enqueued and {depth - 2} host threads build the plans of steps "
-                           f"i+1..i+{depth - 2}") if pipelined
+            "pipelining": (f"rksc_pipeline, {depth} steps in flight: one gate stream, one attention stream (attention "
+                           f"launches back to back in step order, the gates of later steps beside them) and "
+                           f"{max(1, depth - 2)} host thread(s) of the library that build tables and plans; CUDA events "
+                           f"around every step's segment kernels") if pipelined
             else "none (steps strictly serial)",
             "unique_kv_bytes": kv_bytes, "branches": B, "work_items": plan.num_work_items,
             "l2": ("inputs larger than L2 (unique KV %.0f MB vs L2 %.0f MB)" % (kv_bytes / 1e6, l2_bytes / 1e6))

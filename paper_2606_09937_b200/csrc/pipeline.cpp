@@ -239,7 +239,11 @@ extern "C" RKSC_API int32_t rksc_pipeline_create(const rksc_layout* layout, int3
     p->timing = timing != 0;
     bool ok = cudaGetDevice(&p->device) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&p->gate_stream, cudaStreamNonBlocking) == cudaSuccess;
-    ok = ok && cudaStreamCreateWithFlags(&p->att_stream, cudaStreamNonBlocking) == cudaSuccess;
+    // the attention stream outranks the gate stream: where both have thread blocks waiting for an SM,
+    // the persistent attention kernels get it, and the gates of later steps fill what is left
+    int prio_lo = 0, prio_hi = 0;
+    ok = ok && cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithPriority(&p->att_stream, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&p->ev_inputs, cudaEventDisableTiming) == cudaSuccess;
     for (auto& s : p->slots) {
         ok = ok && cudaMalloc(reinterpret_cast<void**>(&s.map_dev), (size_t)B * 4) == cudaSuccess;
