@@ -234,26 +234,61 @@ class Tables:
                 ("seg_block_off", "seg_blocks", "seg_num_tokens", "br_seg_off", "br_segs")}
 
 
+class _OwnedView(np.ndarray):
+    """A view of memory another object owns; ``_owner`` keeps that object alive as long as the view
+    (or anything sliced from it) is."""
+
+
+class LibTables(Tables):
+    """An rksc_tables the library allocated (rksc_tables_from_gate and the other table calls): kept as
+    it is and freed with this object, so that handing it to the next call costs no copy.  The array
+    attributes are views of the library's memory, made on access; each keeps this object alive."""
+
+    _FIELDS = {"seg_block_off": ("num_segments", 1), "seg_num_tokens": ("num_segments", 0),
+               "br_seg_off": ("num_branches", 1)}
+
+    def __init__(self, c: "_CTables"):
+        self.c = c
+
+    def _view(self, name):
+        c = self.c
+        if name in self._FIELDS:
+            count, extra = self._FIELDS[name]
+            n = int(getattr(c, count)) + extra
+        elif name == "seg_blocks":
+            n = int(c.seg_block_off[c.num_segments])
+        else:   # br_segs
+            n = int(c.br_seg_off[c.num_branches])
+        if n <= 0:
+            return np.zeros(0, dtype=np.int32)
+        v = np.ctypeslib.as_array(getattr(c, name), shape=(n,)).view(_OwnedView)
+        v._owner = self
+        return v
+
+    seg_block_off = property(lambda self: self._view("seg_block_off"))
+    seg_blocks = property(lambda self: self._view("seg_blocks"))
+    seg_num_tokens = property(lambda self: self._view("seg_num_tokens"))
+    br_seg_off = property(lambda self: self._view("br_seg_off"))
+    br_segs = property(lambda self: self._view("br_segs"))
+
+    def __del__(self):
+        try:
+            lib().rksc_tables_free(C.byref(self.c))
+        except Exception:
+            pass
+
+
 def rksc_tables_from_gate(branch_to_prefix, num_prefixes,
                           shared_off, shared_pages, shared_ntok,
                           priv_off, priv_pages, priv_ntok,
                           sfx_off, sfx_pages, sfx_ntok) -> Tables:
-    """Host call: segment tables from a gate map (arrays are copied out of the library's result)."""
+    """Host call: segment tables from a gate map (the library's result, wrapped without a copy)."""
     arrs = [_i32(a) for a in (branch_to_prefix, shared_off, shared_pages, shared_ntok,
                               priv_off, priv_pages, priv_ntok, sfx_off, sfx_pages, sfx_ntok)]
     out = _CTables()
     st = lib().rksc_tables_from_gate(len(arrs[0]), int(num_prefixes), *[_p(a) for a in arrs], C.byref(out))
     _check(st, "rksc_tables_from_gate")
-    try:
-        S, B = out.num_segments, out.num_branches
-        cp = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(max(n, 1),))[:n].copy()
-        seg_block_off = cp(out.seg_block_off, S + 1)
-        br_seg_off = cp(out.br_seg_off, B + 1)
-        t = Tables(seg_block_off, cp(out.seg_blocks, int(seg_block_off[-1])), cp(out.seg_num_tokens, S),
-                   br_seg_off, cp(out.br_segs, int(br_seg_off[-1])))
-    finally:
-        lib().rksc_tables_free(C.byref(out))
-    return t
+    return LibTables(out)
 
 
 class Plan:
@@ -463,38 +498,20 @@ def rksc_tables_drop_evicted(tables, evicted) -> Tables:
     out = _CTables()
     st = lib().rksc_tables_drop_evicted(C.byref(t.c), ev.ctypes.data_as(C.c_void_p), C.byref(out))
     _check(st, "rksc_tables_drop_evicted")
-    try:
-        S, B = out.num_segments, out.num_branches
-        cp = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(max(n, 1),))[:n].copy()
-        seg_block_off = cp(out.seg_block_off, S + 1)
-        br_seg_off = cp(out.br_seg_off, B + 1)
-        res = Tables(seg_block_off, cp(out.seg_blocks, int(seg_block_off[-1])), cp(out.seg_num_tokens, S),
-                     br_seg_off, cp(out.br_segs, int(br_seg_off[-1])))
-    finally:
-        lib().rksc_tables_free(C.byref(out))
-    return res
+    return LibTables(out)
 
 
 def rksc_tables_append_token(tables, new_pages):
     """Host call: one decode step on the tables.  Returns (Tables, page int32 [B], slot int32 [B])."""
     t = Tables.of(tables)
-    B = len(t.br_seg_off) - 1
+    B = int(t.c.num_branches)
     npg = _i32(new_pages) if new_pages is not None else None
     page = np.empty(max(B, 1), dtype=np.int32)
     slot = np.empty(max(B, 1), dtype=np.int32)
     out = _CTables()
     st = lib().rksc_tables_append_token(C.byref(t.c), _p(npg) if npg is not None else None, C.byref(out), _p(page), _p(slot))
     _check(st, "rksc_tables_append_token")
-    try:
-        S = out.num_segments
-        cp = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(max(n, 1),))[:n].copy()
-        seg_block_off = cp(out.seg_block_off, S + 1)
-        br_seg_off = cp(out.br_seg_off, B + 1)
-        res = Tables(seg_block_off, cp(out.seg_blocks, int(seg_block_off[-1])), cp(out.seg_num_tokens, S),
-                     br_seg_off, cp(out.br_segs, int(br_seg_off[-1])))
-    finally:
-        lib().rksc_tables_free(C.byref(out))
-    return res, page[:B], slot[:B]
+    return LibTables(out), page[:B], slot[:B]
 
 
 def rksc_kv_append(layout, k_pool, v_pool, k_new, v_new, page, slot, stream=None):
@@ -561,16 +578,7 @@ def rksc_tables_for_suffix_prefill(tables, s: int) -> Tables:
     out = _CTables()
     st = lib().rksc_tables_for_suffix_prefill(C.byref(t.c), int(s), C.byref(out))
     _check(st, "rksc_tables_for_suffix_prefill")
-    try:
-        S, B = out.num_segments, out.num_branches
-        cp = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(max(n, 1),))[:n].copy()
-        seg_block_off = cp(out.seg_block_off, S + 1)
-        br_seg_off = cp(out.br_seg_off, B + 1)
-        res = Tables(seg_block_off, cp(out.seg_blocks, int(seg_block_off[-1])), cp(out.seg_num_tokens, S),
-                     br_seg_off, cp(out.br_segs, int(br_seg_off[-1])))
-    finally:
-        lib().rksc_tables_free(C.byref(out))
-    return res
+    return LibTables(out)
 
 
 def rksc_decode_step_host(layout, h_branch, h_root, cand_prefix, alpha, tau, flat, q, k_pool, v_pool,
