@@ -158,4 +158,57 @@ def test_in_flight_rules_small_mass_buffer_and_timing():
     # without a mass buffer the same pipeline runs the step
     t = small.submit(hb, hr, cand, q, kp, vp, out, None)
     assert small.wait(t).status == 0
+    # destroying a pipeline with steps in flight finishes them first
+    out.fill_(float("nan"))
+    torch.cuda.synchronize()
+    small.submit(hb, hr, cand, q, kp, vp, out, None)
+    small.submit(hb, hr, cand, q, kp, vp, out, None)
     small.close()
+    assert bool(torch.isfinite(out).all())
+
+
+@pytest.mark.gpu
+def test_many_steps_at_full_depth_reuse_their_slots_correctly():
+    """Forty steps eight deep: every slot is reused five times, gates of later steps run beside the
+    attention of earlier ones, and each step's outputs still belong to its own inputs."""
+    import torch
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+    w = workloads.make_config("tiny")
+    depth, n = 8, 40
+    variants = _variants(w, 4)                    # four distinct (query, gate input) pairs, cycled
+    refs = []
+    for s in variants:
+        m_ref, _ = oracle_gate(s.gate)
+        refs.append((m_ref,) + tuple(oracle_attention(s, oracle_tables_from_map(s, m_ref))))
+    L, D = w.gate.h_branch.shape[1:]
+    cap = _mass_capacity(w)
+    pipe = rk.Pipeline(w.layout, w.num_branches, (L, D), w.gate.alpha, w.gate.tau, w.flat, depth=depth,
+                       mass_capacity=cap)
+    kp, vp = w.k_pool.to(dev), w.v_pool.to(dev)
+    hr = w.gate.h_root.to(dev)
+    cand = torch.from_numpy(w.gate.cand_prefix).to(dev)
+    hbs = [s.gate.h_branch.to(dev) for s in variants]
+    qs = [s.q.to(dev) for s in variants]
+    Hq, d = w.layout.num_q_heads, w.layout.head_dim
+    outs = [torch.empty((w.num_branches, Hq, d), dtype=torch.float32, device=dev) for _ in range(depth)]
+    masses = [torch.empty(cap, dtype=torch.float32, device=dev) for _ in range(depth)]
+
+    def check(t, r):
+        m_ref, ref_out, ref_mass = refs[t % 4]
+        assert np.array_equal(r.branch_to_prefix, m_ref), t
+        flat = masses[t % depth].cpu().numpy()
+        ms = [flat[int(r.mass_off[b]) * Hq:int(r.mass_off[b + 1]) * Hq].reshape(Hq, -1) for b in range(w.num_branches)]
+        check_attention(outs[t % depth].cpu().numpy(), ms, ref_out, ref_mass)
+
+    for t in range(n):
+        if t >= depth:
+            check(t - depth, pipe.wait(t - depth))          # before the slot's buffers are reused
+        outs[t % depth].fill_(float("nan"))
+        masses[t % depth].fill_(float("nan"))
+        assert pipe.submit(hbs[t % 4], hr, cand, qs[t % 4], kp, vp, outs[t % depth], masses[t % depth],
+                           after_stream=torch.cuda.current_stream()) == t
+    for t in range(n - depth, n):
+        check(t, pipe.wait(t))
+    pipe.close()
