@@ -99,3 +99,58 @@ def test_config5_long_context_with_holes_full():
     sample = [0, 9, 15]
     ref_out, ref_m = oracle_attention(h, branches=sample)
     check_attention(out, m, ref_out, ref_m, branches=sample)
+
+
+def test_config4_through_the_step_pipeline_as_bench_times_it():
+    """The launch configuration of the headline loop: config 4 through rksc_pipeline, four steps in
+    flight, the same inputs every step.  Every step's map is bit-exact, and the outputs and masses of
+    sampled branches of the first and the last step match the oracle."""
+    import torch
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+    w = workloads.make_config("batched_serving")
+    g, f = w.gate, w.flat
+    B, Hq, d = w.num_branches, w.layout.num_q_heads, w.layout.head_dim
+    m_ref, s_ref = oracle_gate(g)
+    t_ref = oracle_tables_from_map(w, m_ref)
+    cap = 0
+    for b in range(B):
+        r = int(g.cand_prefix[b])
+        cap += max(int(f.shared_off[r + 1] - f.shared_off[r]), int(f.priv_off[b + 1] - f.priv_off[b]))
+        cap += int(f.sfx_off[b + 1] - f.sfx_off[b])
+    cap *= Hq
+    depth, n = 4, 6
+    pipe = rk.Pipeline(w.layout, B, tuple(g.h_branch.shape[1:]), g.alpha, g.tau, f, depth=depth, mass_capacity=cap,
+                       timing=True)
+    hb, hr = g.h_branch.to(dev), g.h_root.to(dev)
+    cand = torch.from_numpy(g.cand_prefix).to(dev)
+    q, kp, vp = w.q.to(dev), w.k_pool.to(dev), w.v_pool.to(dev)
+    outs = [torch.full((B, Hq, d), float("nan"), dtype=torch.float32, device=dev) for _ in range(n)]
+    masses = [torch.full((cap,), float("nan"), dtype=torch.float32, device=dev) for _ in range(n)]
+    torch.cuda.synchronize()
+    res = {}
+    for i in range(n):
+        if i >= depth:
+            res[i - depth] = pipe.wait(i - depth)
+        pipe.submit(hb, hr, cand, q, kp, vp, outs[i], masses[i])
+    for i in range(n - depth, n):
+        res[i] = pipe.wait(i)
+    pipe.close()
+    rng = np.random.default_rng(11)
+    priv = np.flatnonzero(g.built_below_tau)
+    shared = np.flatnonzero(~g.built_below_tau)
+    sample = sorted(set(rng.choice(priv, 4, replace=False).tolist() + rng.choice(shared, 8, replace=False).tolist()))
+    ref_out, ref_m = oracle_attention(w, t_ref, branches=sample)
+    for i in range(n):
+        assert res[i].status == 0 and np.array_equal(res[i].branch_to_prefix, m_ref)
+        assert np.abs(res[i].sigma - s_ref).max() < 1e-5
+        assert res[i].segment_ms > 0.0
+    for i in (0, n - 1):
+        flat = masses[i].cpu().numpy()
+        ms = [None] * B
+        for b in sample:
+            lo, hi = int(res[i].mass_off[b]) * Hq, int(res[i].mass_off[b + 1]) * Hq
+            ms[b] = flat[lo:hi].reshape(Hq, -1)
+        check_attention(outs[i].cpu().numpy(), ms, ref_out, ref_m, branches=sample)
+    assert torch.equal(outs[0], outs[n - 1])      # same inputs, same plan, same arithmetic
