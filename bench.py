@@ -489,6 +489,8 @@ def run_ours(args):
         info["what"] = ("after a step, outside the timed region: rksc_rsbcm_page_scores over the step's block masses, "
                         "then rksc_rsbcm_evict down to the paper's default capacity of 2000 entries")
         line["rsbcm"] = info
+        if batch.has_gate:
+            line["stages"] = stage_times(rk, batch, flush)
         if not args.no_e2e and batch.has_gate:
             line["e2e"] = run_e2e(rk, batch, kv_bytes, args.e2e_steps)
         if not args.no_sweep:
@@ -591,6 +593,38 @@ def _event_us(fn, iters=20):
     e1.record()
     torch.cuda.synchronize()
     return e0.elapsed_time(e1) * 1e3 / iters
+
+
+def stage_times(rk, batch: "DeviceBatch", flush, iters: int = 12):
+    """The stages of a step one by one, outside the timed region: the gate kernel (device time after a
+    write-flush of L2), the copy of its map to the host, and tables + plan on the host (wall time of
+    rksc_plan_create_from_gate, which ends with the upload of the plan's arrays)."""
+    import torch
+    g = batch.w.gate
+    gate_us, copy_us, plan_us = [], [], []
+    for _ in range(iters):
+        flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        rk.rksc_asks_gate(batch.h_branch, batch.h_root, batch.cand, g.alpha, g.tau,
+                          branch_to_prefix=batch.map_dev, sigma=batch.sigma_dev)
+        e1.record()
+        e1.synchronize()
+        gate_us.append(e0.elapsed_time(e1) * 1e3)
+        t0 = time.perf_counter()
+        batch.map_host.copy_(batch.map_dev, non_blocking=False)
+        t1 = time.perf_counter()
+        plan = rk.rksc_plan_create_from_gate(batch.layout, batch.map_host.numpy(), batch.lists)
+        t2 = time.perf_counter()
+        copy_us.append((t1 - t0) * 1e6)
+        plan_us.append((t2 - t1) * 1e6)
+        del plan
+    med = lambda v: statistics.median(v[2:])
+    gate_bytes = (batch.h_branch.numel() + batch.h_root.numel()) * 4
+    return {"gate_kernel_us": med(gate_us), "gate_gbs": gate_bytes / (med(gate_us) * 1e-6) / 1e9,
+            "gate_bytes": gate_bytes, "map_to_host_us": med(copy_us), "tables_and_plan_host_us": med(plan_us),
+            "what": "each stage alone, outside the timed region: gate kernel after a write-flush of L2 (CUDA events), "
+                    "blocking copy of the map (host wall time), rksc_plan_create_from_gate (host wall time)"}
 
 
 def rsbcm_pass(rk, batch: DeviceBatch, plan, mass, entries: slice, capacity: int, timed: bool = True):
