@@ -45,7 +45,7 @@ WORKLOAD_LABEL = {
                        "suffix U[128,1024], 28q/4kv d128, 30% of branches below tau",
     "long_context": "configs[4] long context with eviction holes: 16 branches, prefix 32768 (20% of pages "
                     "evicted) + suffix 2048, 32q/8kv d128",
-    "diverse_phrasing": "diverse-phrasing regime (not a BASELINE config): 15 problems x 8 phrasings at 4 divergence "
+    "diverse_phrasing": "diverse-phrasing regime (an extra workload beside the five configurations): 15 problems x 8 phrasings at 4 divergence "
                         "levels, prefix 512, suffix U[16,144], 28q/4kv d128, alpha 1.5, tau 0.82; the gate shares "
                         "the identical and the minor-rewording phrasings",
 }
