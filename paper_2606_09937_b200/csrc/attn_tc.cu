@@ -783,7 +783,15 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             const bool have_self = citem > 0;                 // warpgroup-uniform
             const bool have_oth = ngroups - citem > 0;        // the other warpgroup had a slot
             if (have_self) {
-                TCP_WAIT(4, wait_or_abort(bar(kBarODone + wg), (uint32_t)(c - 1) & 1u));
+                // O is read out once the P V of this warpgroup's last two slots have completed.  A wait on a
+                // barrier's parity tells the current phase only from the one before it, and nothing orders the
+                // softmax of the last slot after the P V of the slot before it (the barrier that counts every
+                // P V could still be two phases back and let a wait for "the last one" through at once).  The
+                // per-buffer barriers cannot be that far back: the scores of slot c - 1 (c - 2) were only
+                // computed after P V of slot c - 3 (c - 4) had left their buffer.
+                if (c >= 2) TCP_WAIT(4, wait_or_abort(bar(kBarPVDone + wg * 2 + ((c - 2) & 1)), (uint32_t)((c - 2) >> 1) & 1u));
+                if (*s_abort) break;
+                TCP_WAIT(4, wait_or_abort(bar(kBarPVDone + wg * 2 + ((c - 1) & 1)), (uint32_t)((c - 1) >> 1) & 1u));
                 if (*s_abort) break;
                 tc_fence_after();
             }
