@@ -51,6 +51,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t n) {   // n arrivals at once
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -81,6 +84,19 @@ __device__ __forceinline__ bool mbar_try_wait_sleep(uint32_t bar, uint32_t parit
         "}\n"
         : "=r"(ok)
         : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {   // never blocks
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
 }
@@ -184,7 +200,7 @@ struct SmemLayout {
     static constexpr int kScrOff = kRing;
     static constexpr int kMlOff = kScrOff + kCW * kScrWarp;   // m[4][16], l[4][16]
     static constexpr int kBarOff = kMlOff + 2 * kCW * 16 * 4;  // full[kNS], empty[kNS]
-    static constexpr int kHdrOff = kBarOff + ((3 * kNS * 8 + 8 + 15) / 16) * 16;  // after the barriers: full, empty, consumers' own, header ready
+    static constexpr int kHdrOff = kBarOff + ((4 * kNS * 8 + 8 + 15) / 16) * 16;  // after the barriers: full, empty, consumers' own, header ready, partials ready
     static_assert(kBarOff % 8 == 0 && kHdrOff % 16 == 0 && kScrOff % 16 == 0, "shared-memory alignment");
     static constexpr int kPagesOff = kHdrOff + kNS * 64;       // one SlotHeader per slot, then its page ids
     static constexpr int kFlagOff = kPagesOff + kNS * kSP * 4;
@@ -207,6 +223,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     const uint32_t bar_empty = bar_full + kNS * 8;
     const uint32_t bar_cons = bar_empty + kNS * 8;   // the four consumer warps meet here in the item epilogue
     const uint32_t bar_hdr = bar_cons + 8;           // [kNS] header and page ids of the slot written (K producer -> V producer)
+    const uint32_t bar_epi = bar_hdr + kNS * 8;      // [kNS] a small-row item's page-lane states are in this slot's memory (consumers -> V producer)
     SlotHeader* s_hdr = reinterpret_cast<SlotHeader*>(smem + SL::kHdrOff);
     int32_t* s_pages = reinterpret_cast<int32_t*>(smem + SL::kPagesOff);
     volatile int32_t* s_abort = reinterpret_cast<volatile int32_t*>(smem + SL::kFlagOff);
@@ -217,6 +234,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             mbar_init(bar_full + 8 * i, 2);     // the K and the V producer
             mbar_init(bar_empty + 8 * i, kCW);
             mbar_init(bar_hdr + 8 * i, 1);
+            mbar_init(bar_epi + 8 * i, kCW);
         }
         mbar_init(bar_cons, kCW);
         *s_abort = 0;
@@ -338,19 +356,82 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         // One warp cannot issue TMA copies fast enough for a CTA's share of the memory bandwidth: this
         // one follows the K producer slot by slot (header and page ids through shared memory) and
         // issues the V half of every slot.
+        // It also finishes the small-row items (<= 8 stacked rows: the four consumer warps were four page
+        // lanes of the same rows): the consumers leave their lane states in the memory of the item's
+        // last slot, signal bar_epi and go on to the next item; this warp, which waits most of the
+        // time, merges the lanes, writes the partial result and releases the slot.
         const uint64_t kv_policy = l2_evict_first_policy();
+        uint32_t pending = 0;    // ring slots that hold such lane states (or will, once the consumers get there)
+        uint32_t epi_par = 0;    // per ring slot: parity of its next bar_epi phase
+        auto finish_item = [&](int slot) {
+            constexpr int RS = HD + 4, CPL = HD / 32;   // row stride of a lane's O^T, columns per thread here
+            const WorkItem w = s_hdr[slot].it;
+            const int nrows = w.num_sharers * a.G;
+            const size_t prow0 = (size_t)w.part_row_base;
+            const float* base = reinterpret_cast<const float*>(smem + slot * SL::kSlot);
+            for (int row = 0; row < nrows; ++row) {
+                float mw[kCW], M = -INFINITY;
+#pragma unroll
+                for (int p = 0; p < kCW; ++p) {
+                    mw[p] = base[p * (SL::kPage / 4) + 8 * RS + row];
+                    M = fmaxf(M, mw[p]);
+                }
+                float lsum = 0.f, acc[CPL];
+#pragma unroll
+                for (int c = 0; c < CPL; ++c) acc[c] = 0.f;
+#pragma unroll
+                for (int p = 0; p < kCW; ++p) {
+                    const float* wl = base + p * (SL::kPage / 4);
+                    const float wt = (mw[p] == -INFINITY) ? 0.f : fast_exp2(mw[p] - M);
+                    lsum += wt * wl[8 * RS + 8 + row];
+#pragma unroll
+                    for (int c = 0; c < CPL; ++c) acc[c] += wt * wl[row * RS + CPL * lane + c];
+                }
+                float* dst = a.part_o + (prow0 + row) * HD + CPL * lane;
+#pragma unroll
+                for (int c = 0; c < CPL; ++c) dst[c] = acc[c] / lsum;
+                if (lane == 0) a.part_lse[prow0 + row] = M + fast_log2(lsum);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_n(bar_empty + 8 * slot, kCW);   // in the consumers' stead
+            pending &= ~(1u << slot);
+            epi_par ^= 1u << slot;
+        };
         for (int seq = 0; !*s_abort; ++seq) {
             const int slot = seq % kNS;
+            // The K producer cannot publish this ring slot again before the item that ended in it is
+            // finished: do that first.  The other slots are looked at in passing.
+#pragma unroll
+            for (int s2 = 0; s2 < kNS; ++s2) {
+                if (!(pending & (1u << s2))) continue;
+                const uint32_t par = (epi_par >> s2) & 1u;
+                if (s2 == slot) {
+                    wait_or_abort(bar_epi + 8 * s2, par);
+                    if (*s_abort) break;
+                    finish_item(s2);
+                } else if (__all_sync(0xffffffffu, mbar_test(bar_epi + 8 * s2, par))) {
+                    finish_item(s2);
+                }
+            }
+            if (*s_abort) break;
             wait_or_abort(bar_hdr + 8 * slot, (uint32_t)(seq / kNS) & 1u);
             if (*s_abort) break;
             const int item = s_hdr[slot].item;
             const uint32_t bar = bar_full + 8 * slot;
             if (item < 0) {
                 if (lane == 0) mbar_arrive(bar);
+                // the items still to be finished
+#pragma unroll
+                for (int s2 = 0; s2 < kNS; ++s2) {
+                    if (!(pending & (1u << s2)) || *s_abort) continue;
+                    wait_or_abort(bar_epi + 8 * s2, (epi_par >> s2) & 1u);
+                    if (!*s_abort) finish_item(s2);
+                }
                 break;
             }
             const int npg = s_hdr[slot].num_pages;
             const int kvh = s_hdr[slot].it.kv_head;
+            const bool ends_small = s_hdr[slot].last && s_hdr[slot].it.num_sharers * a.G <= 8;
             const int page = s_pages[slot * kSP + (lane & (kSP - 1))];
             __syncwarp();
             if (lane == 0) mbar_arrive_expect_tx(bar, npg * SL::kTile);
@@ -361,6 +442,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 #pragma unroll
                 for (int hh = 0; hh < HD / 64; ++hh) tma_load_2d(dst + hh * 2048, &tm_v, hh * 64, y, bar, kv_policy);
             }
+            if (ends_small) pending |= 1u << slot;
         }
         return;
     }
@@ -675,27 +757,9 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 mine[8 * RS + 8 + 2 * t] = l0;
                 mine[8 * RS + 8 + 2 * t + 1] = l1;
             }
-            consumer_sync();
-            if (*s_abort) break;
-            for (int idx = tid; idx < rows * HD; idx += kCW * 32) {
-                const int row = idx / HD, col = idx % HD;
-                float M = -INFINITY;
-#pragma unroll
-                for (int p = 0; p < kCW; ++p) M = fmaxf(M, base[p * (SL::kPage / 4) + 8 * RS + row]);
-                float lsum = 0.f, acc = 0.f;
-#pragma unroll
-                for (int p = 0; p < kCW; ++p) {
-                    const float* w = base + p * (SL::kPage / 4);
-                    const float mw = w[8 * RS + row];
-                    const float wt = (mw == -INFINITY) ? 0.f : fast_exp2(mw - M);
-                    lsum += wt * w[8 * RS + 8 + row];
-                    acc += wt * w[row * RS + col];
-                }
-                a.part_o[(prow0 + row) * HD + col] = acc / lsum;
-                if (col == 0) a.part_lse[prow0 + row] = M + fast_log2(lsum);
-            }
+            // the V producer warp merges the four lanes, writes the partial and releases the slot
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_empty + 8 * slot);   // this warp no longer reads the slot
+            if (lane == 0) mbar_arrive(bar_epi + 8 * slot);
         } else if (PL == 1) {
             // one warp per row tile: straight from registers
             if (active) {
