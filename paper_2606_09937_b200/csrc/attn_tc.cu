@@ -802,11 +802,16 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             if (*s_abort) break;
             tc_fence_after();
             {
+                // The two warpgroups hold the item's even and odd slots; which of them holds which depends on
+                // how many slots this CTA ran before the item (items are claimed dynamically).  The two states
+                // are therefore combined symmetrically - products rounded on their own, then one addition, no
+                // fused multiply-add across the two - so that an item's partial result has the same bits
+                // whichever CTA ran it after whatever.
                 const float2 oth = s_ml[((k & 1) * 2 + (1 - wg)) * 128 + row];
                 const float M = fmaxf(have_self ? m : -INFINITY, have_oth ? oth.x : -INFINITY);
                 const float w_self = have_self ? fast_exp2(m - M) : 0.f;
                 const float w_oth = have_oth ? fast_exp2(oth.x - M) : 0.f;
-                const float L = w_self * l + w_oth * oth.y;
+                const float L = __fadd_rn(__fmul_rn(w_self, l), __fmul_rn(w_oth, oth.y));
                 const float inv = 1.f / L;
                 const float c_self = w_self * inv, c_oth = w_oth * inv;
                 float* dst = a.part_o + ((size_t)it_part_row_base + row) * HD + wg * 64;
@@ -818,10 +823,10 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     tmem_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        float v = 0.f;
-                        if (have_self) v = c_self * __uint_as_float(os[j]);
-                        if (have_oth) v += c_oth * __uint_as_float(oo[j]);
-                        os[j] = __float_as_uint(v);
+                        // both products rounded, then one addition: the same bits in either role
+                        const float ps_ = have_self ? __fmul_rn(c_self, __uint_as_float(os[j])) : 0.f;
+                        const float po_ = have_oth ? __fmul_rn(c_oth, __uint_as_float(oo[j])) : 0.f;
+                        os[j] = __float_as_uint(__fadd_rn(ps_, po_));
                     }
                     if (valid) {
 #pragma unroll

@@ -187,3 +187,32 @@ def test_repeated_calls_are_bitwise_identical_on_a_poisoned_workspace(name, call
         else:
             assert torch.equal(out, ref[0]), f"call {i}: outputs differ by {float((out - ref[0]).abs().max())}"
             assert torch.equal(mass, ref[1]), f"call {i}: masses differ"
+
+
+def test_suffix_prefill_calls_are_bitwise_identical_whichever_cta_takes_which_item():
+    """Many tensor-core items per CTA, claimed dynamically: the two warpgroups of a CTA split an item's
+    slots by the parity of the CTA's running slot count, so an item may find them in either role; the
+    item epilogue combines their states symmetrically, and the result has the same bits every time."""
+    import torch
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+    w = workloads.make_config("qwen_layer")
+    m_ref, _ = oracle_gate(w.gate)
+    vt = rk.rksc_tables_for_suffix_prefill(oracle_tables_from_map(w, m_ref), 16)
+    plan = rk.rksc_plan_create(w.layout, vt)
+    assert plan.num_work_items > 2 * 148          # more items than CTAs: some CTA runs several
+    g = torch.Generator().manual_seed(5)
+    q = torch.randn((plan.num_branches, w.layout.num_q_heads, w.layout.head_dim), generator=g).to(torch.bfloat16).to(dev)
+    kp, vp = w.k_pool.to(dev), w.v_pool.to(dev)
+    ws = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device=dev)
+    ref = None
+    for i in range(60):
+        ws.fill_(0xFF)
+        out, mass, status = rk.rksc_branch_decode_attention(plan, q, kp, vp, workspace=ws)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        if ref is None:
+            ref = (out, mass)
+        else:
+            assert torch.equal(out, ref[0]) and torch.equal(mass, ref[1]), f"call {i}"
