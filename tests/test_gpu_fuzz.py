@@ -1,0 +1,59 @@
+"""Seeded random segment structures through the attention path against the oracle.
+
+Each case draws heads (Hkv in 1..8, group size 1..8), head_dim 64 or 128, up to 39 branches, up to
+three shared segments with random sharer sets and a private segment per branch, token counts either
+uniform or from a list of values around the page, slot and tile sizes (1, 15, 16, 17, ..., 257), and
+a query gain of 1, 3 or 8 (sharper softmax).  Both kernels, every row-count class and ragged last
+pages come up; outputs and block masses must meet the path's tolerances in every case.
+"""
+import numpy as np
+import pytest
+
+import workloads
+from helpers import check_attention, oracle_attention
+
+pytestmark = pytest.mark.gpu
+
+EDGE = [1, 2, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256, 257]
+
+
+def _case(seed):
+    rng = np.random.default_rng(seed)
+    hd = int(rng.choice([64, 128, 128, 128]))
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.choice([1, 2, 4, 7, 8]))
+    B = int(rng.integers(1, 40))
+    seg_ntok, br = [], [[] for _ in range(B)]
+    for s in range(int(rng.integers(0, 4))):
+        seg_ntok.append(int(rng.choice(EDGE)) if rng.random() < 0.5 else int(rng.integers(1, 700)))
+        for b in rng.choice(B, size=int(rng.integers(1, B + 1)), replace=False):
+            br[int(b)].append(s)
+    for b in range(B):
+        if rng.random() < 0.85 or not br[b]:
+            n = int(rng.choice(EDGE)) if rng.random() < 0.5 else int(rng.integers(0, 300))
+            if n == 0 and not br[b] and rng.random() < 0.7:
+                n = 5
+            seg_ntok.append(n)
+            br[b].append(len(seg_ntok) - 1)
+        br[b] = sorted(br[b])
+    gain = float(rng.choice([1.0, 1.0, 3.0, 8.0]))
+    return workloads.make_from_segments(f"fuzz{seed}", Hkv * G, Hkv, hd, seg_ntok, br, seed=1000 + seed, q_gain=gain)
+
+
+@pytest.mark.parametrize("first", [0, 40, 80])
+def test_random_segment_structures_match_the_oracle(first):
+    import torch
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+    for seed in range(first, first + 40):
+        w = _case(seed)
+        plan = rk.rksc_plan_create(w.layout, w.tables)
+        out, mass, status = rk.rksc_branch_decode_attention(plan, w.q.to(dev), w.k_pool.to(dev), w.v_pool.to(dev))
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, seed
+        ref_out, ref_m = oracle_attention(w)
+        try:
+            check_attention(out.cpu().numpy(), rk.split_block_mass(plan, mass), ref_out, ref_m)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from None
