@@ -289,6 +289,11 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     volatile int32_t* s_abort = reinterpret_cast<volatile int32_t*>(smem + kFlagOff);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // The CTA's first item is item blockIdx.x.  The two warps that need it first ask for it before
+    // anything else, so that the round trip passes behind the set-up below (the plan's arrays are
+    // written by no kernel: reading them does not have to wait for the kernel before this one).
+    WorkItem it_first{};
+    if ((warp == kProducerWarp || warp == kQWarp) && (int)blockIdx.x < a.num_tc_items) it_first = a.plan.items[blockIdx.x];
     if (tid == 0) {
         for (int i = 0; i < kNK; ++i) {
             mbar_init(bar(kBarFullK + i), 1);
@@ -397,7 +402,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const uint64_t kv_policy = l2_evict_first_policy();
         int seq = 0;
         int idx = (int)blockIdx.x;
-        WorkItem it = fetch_item(idx);
+        WorkItem it = it_first;
         publish(idx, it);
         int ids = fetch_ids(it, 0);
         while (idx < a.num_tc_items && !*s_abort) {
@@ -487,8 +492,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const int G = a.G;
         // the CTA's first item is item blockIdx.x: fetched here, alongside the producer's own fetch,
         // so that its sharers and query rows are on their way before the producer has published it
-        WorkItem it0{};
-        if ((int)blockIdx.x < a.num_tc_items) it0 = a.plan.items[blockIdx.x];
+        const WorkItem it0 = it_first;
         for (int k = 0; !*s_abort; ++k) {
             const int e = k % kNI;
             Sharer sh[4];
