@@ -216,3 +216,38 @@ def test_suffix_prefill_calls_are_bitwise_identical_whichever_cta_takes_which_it
             ref = (out, mass)
         else:
             assert torch.equal(out, ref[0]) and torch.equal(mass, ref[1]), f"call {i}"
+
+
+def test_two_plans_on_two_streams_at_once_give_their_single_stream_bits():
+    """Distinct plans on distinct streams may run at the same time (the header's promise): their persistent
+    kernels then share the SMs, and each call must still give exactly what it gives alone."""
+    import torch
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+
+    def prepare(name):
+        w = workloads.make_config(name)
+        t = w.tables if w.tables is not None else oracle_tables_from_map(w, oracle_gate(w.gate)[0])
+        plan = rk.rksc_plan_create(w.layout, t)
+        x = dict(plan=plan, q=w.q.to(dev), kp=w.k_pool.to(dev), vp=w.v_pool.to(dev),
+                 ws=torch.empty(plan.workspace_bytes, dtype=torch.uint8, device=dev))
+        out, mass, status = rk.rksc_branch_decode_attention(plan, x["q"], x["kp"], x["vp"], workspace=x["ws"])
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        x["ref"] = (out.clone(), mass.clone())
+        return x
+
+    pair = [prepare("tot"), prepare("diverse_phrasing")]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for i in range(30):
+        res = []
+        for x, s in zip(pair, streams):
+            with torch.cuda.stream(s):
+                x["ws"].fill_(0xFF)
+                res.append(rk.rksc_branch_decode_attention(x["plan"], x["q"], x["kp"], x["vp"], workspace=x["ws"],
+                                                           stream=s))
+        torch.cuda.synchronize()
+        for x, (out, mass, status) in zip(pair, res):
+            assert int(status.item()) == 0
+            assert torch.equal(out, x["ref"][0]) and torch.equal(mass, x["ref"][1]), f"round {i}"
