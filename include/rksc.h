@@ -48,6 +48,14 @@ RKSC_API const char* rksc_strerror(int32_t status);
 /* Text of the CUDA error behind the calling thread's most recent RKSC_ERR_CUDA from a launch. */
 RKSC_API const char* rksc_last_cuda_error(void);
 
+/* Self-test of the bounded-wait mechanism every kernel of this library uses: launches one small CTA
+ * whose warps wait on a shared-memory barrier that nothing ever completes, with a limit of
+ * `limit_cycles` SM cycles (the production kernels' limit is 2^32).  When the limit runs out the
+ * waiting warps record RKSC_ERR_DEVICE_TIMEOUT in *device_status (dev int32, zeroed by the caller),
+ * stop waiting and the kernel returns normally: the context stays usable and nothing traps.
+ * limit_cycles in [1, 2^31].  Asynchronous on `stream`. */
+RKSC_API int32_t rksc_debug_wait_timeout(int64_t limit_cycles, int32_t* device_status, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * ASKS similarity gate  (paper Eq. 2 and Algorithm 2)
  *

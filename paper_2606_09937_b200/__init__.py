@@ -32,6 +32,7 @@ from .binding import (  # noqa: F401
     rksc_cgee_logit_entropy,
     rksc_cgee_entropy_exit,
     rksc_cgee_verify_skip,
+    rksc_debug_wait_timeout,
     Pipeline,
     StepResult,
     STATIC_WORKSPACE_BYTES,

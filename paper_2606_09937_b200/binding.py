@@ -42,6 +42,7 @@ EXPORTED_SYMBOLS = (
     "rksc_cgee_logit_entropy",
     "rksc_cgee_entropy_exit",
     "rksc_cgee_verify_skip",
+    "rksc_debug_wait_timeout",
     "rksc_pipeline_create",
     "rksc_pipeline_submit",
     "rksc_pipeline_wait",
@@ -151,6 +152,8 @@ def lib() -> C.CDLL:
     L.rksc_tables_for_suffix_prefill.argtypes = [C.POINTER(_CTables), C.c_int32, C.POINTER(_CTables)]
     L.rksc_tables_drop_evicted.restype = C.c_int32
     L.rksc_tables_drop_evicted.argtypes = [C.POINTER(_CTables), C.c_void_p, C.POINTER(_CTables)]
+    L.rksc_debug_wait_timeout.restype = C.c_int32
+    L.rksc_debug_wait_timeout.argtypes = [C.c_int64, C.c_void_p, C.c_void_p]
     L.rksc_pipeline_create.restype = C.c_int32
     L.rksc_pipeline_create.argtypes = ([C.POINTER(_CLayout)] + [C.c_int32] * 4 + [C.c_float, C.c_float] + [i32p] * 9 +
                                        [C.c_int32, C.c_int64, C.c_int32, C.POINTER(C.c_void_p)])
@@ -607,6 +610,13 @@ def rksc_decode_step_host(layout, h_branch, h_root, cand_prefix, alpha, tau, fla
         block_mass.numel() if block_mass is not None else 0, mo, _stream_ptr(stream, k_pool.device))
     _check(st, "rksc_decode_step_host")
     return st
+
+
+def rksc_debug_wait_timeout(limit_cycles: int, device_status, stream=None) -> int:
+    """Self-test of the kernels' bounded wait (see rksc.h); returns the host status of the launch."""
+    return int(lib().rksc_debug_wait_timeout(int(limit_cycles), device_status.data_ptr() if device_status is not None
+                                             else None, _stream_ptr(stream, device_status.device if device_status
+                                                                    is not None else None)))
 
 
 class StepResult:

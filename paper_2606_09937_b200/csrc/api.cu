@@ -800,3 +800,20 @@ extern "C" RKSC_API int32_t rksc_kv_append(const rksc_layout* layout, void* k_po
     }
     return RKSC_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded wait
+// ---------------------------------------------------------------------------------------------
+
+extern "C" RKSC_API int32_t rksc_debug_wait_timeout(int64_t limit_cycles, int32_t* device_status, void* stream) {
+    if (limit_cycles < 1 || limit_cycles > ((int64_t)1 << 31) || !device_status) return RKSC_ERR_INVALID_ARG;
+    int32_t st = ensure_device(nullptr);
+    if (st != RKSC_OK) return st;
+    const cudaError_t e = launch_wait_timeout((long long)limit_cycles, device_status, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda = e;
+        cudaGetLastError();
+        return RKSC_ERR_CUDA;
+    }
+    return RKSC_OK;
+}

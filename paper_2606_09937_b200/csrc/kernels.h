@@ -63,4 +63,6 @@ cudaError_t launch_kv_append(void* k_pool, void* v_pool, const void* k_new, cons
 cudaError_t launch_rsbcm_select(const double* score, const int32_t* depth, int32_t n, uint32_t k, uint64_t* keys,
                                 uint8_t* evicted, int32_t* num_evicted, cudaStream_t stream);
 
+cudaError_t launch_wait_timeout(long long limit_cycles, int32_t* status, cudaStream_t stream);
+
 }  // namespace rksc

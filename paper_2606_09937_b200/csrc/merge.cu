@@ -165,4 +165,52 @@ cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream) {
     return cudaLaunchKernelEx(&cfg, merge_kernel, a, wpk_log2);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded wait (rksc_debug_wait_timeout): same structure as the kernels' waits -
+// try_wait with a suspend hint in a loop, the SM cycle counter as the limit, an abort flag in shared
+// memory that makes every later wait of the CTA return at once, the status word written once.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+__global__ void __launch_bounds__(128) wait_timeout_kernel(long long limit, int32_t* status) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    const uint32_t b = static_cast<uint32_t>(__cvta_generic_to_shared(&bar));
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b) : "memory");   // one arrival expected, none comes
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    for (int round = 0; round < 3; ++round) {     // after the first expiry the later waits return at once
+        if (*reinterpret_cast<volatile int*>(&abort_flag)) break;
+        const long long t0 = clock64();
+        for (;;) {
+            uint32_t ok;
+            asm volatile(
+                "{\n"
+                ".reg .pred p;\n"
+                "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+                "selp.u32 %0, 1, 0, p;\n"
+                "}\n"
+                : "=r"(ok)
+                : "r"(b), "r"(0u), "r"(1000u)
+                : "memory");
+            if (ok) break;
+            if (clock64() - t0 > limit) {
+                abort_flag = 1;
+                if (status) atomicExch(status, RKSC_ERR_DEVICE_TIMEOUT);
+                break;
+            }
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_wait_timeout(long long limit, int32_t* status, cudaStream_t stream) {
+    wait_timeout_kernel<<<1, 128, 0, stream>>>(limit, status);
+    return cudaGetLastError();
+}
+
 }  // namespace rksc
