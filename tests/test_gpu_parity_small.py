@@ -86,6 +86,39 @@ def test_long_segment_many_chunks_and_custom_scale():
     assert plan.num_work_items > 8
 
 
+@pytest.mark.parametrize("sharers", [1, 24])
+def test_very_long_context_against_the_closed_form(sharers):
+    """262 144 tokens (16 384 pages, 32 chunks at the 512-page item cap) with identical keys: every score is
+    equal, so out = mean of V and every full block holds 16 / T of the mass, whatever the queries - a
+    definition the oracle is not needed for at this size.  One branch alone runs the warp path over many
+    chunks; 24 sharers x 4 heads run the tensor-core path (96 stacked rows)."""
+    import torch
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+    T, Hkv, G, d = 262144, 1, 4, 128
+    w = workloads.make_from_segments("maxlen", Hkv * G, Hkv, d, [T], [[0]] * sharers, seed=21)
+    key = torch.randn(d, generator=torch.Generator().manual_seed(3)).to(torch.bfloat16)
+    pages = torch.from_numpy(np.asarray(w.tables.seg_blocks, dtype=np.int64))
+    k_pool = w.k_pool.clone()
+    k_pool[pages] = key                                   # the same key in every slot of every listed page
+    plan = rk.rksc_plan_create(w.layout, w.tables)
+    assert plan.num_work_items >= 32
+    out, mass, status = rk.rksc_branch_decode_attention(plan, w.q.to(dev), k_pool.to(dev), w.v_pool.to(dev))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    v_mean = w.v_pool[pages].to(torch.float64).mean(dim=(0, 2)).numpy()          # [Hkv][d]
+    got = out.cpu().numpy().astype(np.float64)
+    diff = got - v_mean[0][None, None, :]
+    assert np.abs(diff).max() <= 2e-4                                            # |mean| ~ 2e-3 per element
+    rel = np.linalg.norm(diff, axis=-1) / np.linalg.norm(v_mean[0])
+    assert rel.max() <= 1e-2, rel.max()                                          # the relative criterion binds here
+    m = rk.split_block_mass(plan, mass)
+    for b in range(sharers):
+        assert np.abs(m[b].astype(np.float64) - 16.0 / T).max() <= 1e-7
+        assert np.abs(m[b].astype(np.float64).sum(axis=1) - 1.0).max() <= 1e-5
+
+
 def test_tot_small():
     w = workloads.make_tot(root_tokens=300, level_tokens=50)
     _parity(w)
