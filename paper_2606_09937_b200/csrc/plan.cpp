@@ -139,11 +139,14 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     const int cap = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, fair * 2 / 3));
     const int base = (int)std::min<int64_t>(128, std::max<int64_t>(kMinChunk, fair / 6));
 
-    // Items of the tensor-core kernel are as long as three quarters of an SM's share of ALL the work:
-    // that kernel pays for every item (epilogue, hand-over) and once per CTA at its start, and the
-    // warp-MMA kernel, which starts on each SM as the tensor-core CTA there ends, takes up the slack
-    // of an uneven split.
-    const int tc_chunk = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, fair * 3 / 2));
+    // Items of the tensor-core kernel are as long as an SM's share of ALL the work (twice a CTA's share
+    // at two warp-kernel CTAs per SM): that kernel pays for every item (epilogue, hand-over) and once
+    // per CTA at its start, and the warp-MMA kernel, which starts at once on the SMs the tensor-core
+    // kernel leaves free and on each of the others as the tensor-core CTA there ends, takes up the
+    // slack of an uneven split.  Measured over long-context shapes (8 k - 64 k shared prefix, 8 - 32
+    // branches) this length was the best of 1 x ... 3 x a CTA's share (8 % better than 1.5 x), and
+    // neutral on the other configurations.
+    const int tc_chunk = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, fair * 2));
     int64_t rows_total = 0;
     {
         size_t n_items = 0;   // exact count, so that the item vector is allocated once
