@@ -48,6 +48,9 @@ WORKLOAD_LABEL = {
     "diverse_phrasing": "diverse-phrasing regime (an extra workload beside the five configurations): 15 problems x 8 phrasings at 4 divergence "
                         "levels, prefix 512, suffix U[16,144], 28q/4kv d128, alpha 1.5, tau 0.82; the gate shares "
                         "the identical and the minor-rewording phrasings",
+    "long_prefix_serving": "batched serving with long prefixes (an extra workload beside the five configurations): 32 "
+                           "problems x 8 branches, prefix U[4096,16384], suffix U[16,128], 28q/4kv d128, 30% of "
+                           "branches below tau",
 }
 
 
@@ -147,7 +150,7 @@ class ClockSampler:
 def load_workload(name: str, seed_shift: int = 0):
     import workloads
     base = {"tiny": 0, "qwen_layer": 1, "tot": 2, "batched_serving": 3, "long_context": 4,
-            "diverse_phrasing": 5}[name]
+            "diverse_phrasing": 5, "long_prefix_serving": 6}[name]
     return workloads.make_config(name, seed=workloads.generators.SEED_BASE + base + 1000 * seed_shift)
 
 

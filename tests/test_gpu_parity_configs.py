@@ -251,3 +251,18 @@ def test_two_plans_on_two_streams_at_once_give_their_single_stream_bits():
         for x, (out, mass, status) in zip(pair, res):
             assert int(status.item()) == 0
             assert torch.equal(out, x["ref"][0]) and torch.equal(mass, x["ref"][1]), f"round {i}"
+
+
+def test_long_prefix_serving_sampled():
+    """The larger batch the bench also times (2.4 GB of unique KV: prefixes of 4096-16384 tokens, short
+    suffixes): gate map and tables bit-exact, sampled branches against the oracle, properties for all."""
+    w = workloads.make_config("long_prefix_serving")
+    t = _gate_and_tables(w)
+    out, m, plan = cuda_attention(w, t)
+    _all_branch_properties(out, m)
+    rng = np.random.default_rng(5)
+    priv = np.flatnonzero(w.gate.built_below_tau)
+    shared = np.flatnonzero(~w.gate.built_below_tau)
+    sample = sorted(set(rng.choice(priv, 3, replace=False).tolist() + rng.choice(shared, 5, replace=False).tolist()))
+    ref_out, ref_m = oracle_attention(w, t, branches=sample)
+    check_attention(out, m, ref_out, ref_m, branches=sample)

@@ -524,6 +524,12 @@ def make_config(name: str, **kw) -> Workload:
         return make_long_context(**kw)
     if name == "diverse_phrasing":
         return make_diverse_phrasing(**kw)
+    if name == "long_prefix_serving":
+        # batched serving with prefixes of 4096-16384 tokens and the paper's short suffixes (s = 16 plus up to
+        # 112 decoded tokens): about 2 GB of unique KV, most of it prefixes
+        w = make_batched_serving(prefix_range=(4096, 16384), suffix_range=(16, 128), **kw)
+        w.name = "long_prefix_serving"
+        return w
     raise ValueError(f"unknown config {name!r}; choose from {CONFIG_NAMES}")
 
 
