@@ -35,7 +35,7 @@ FALLBACK_HBM_GBS = 6650.0    # used only when MEASURED_PEAKS.json is absent
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the segment kernel, from the ncu
 # capture summarised under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {"batched_serving": 766851328}   # profiles/seg_attention_batched_serving.md
+NCU_TRAFFIC_BYTES = {"batched_serving": 767356672}   # profiles/seg_attention_batched_serving.md
 
 WORKLOAD_LABEL = {
     "tiny": "configs[0] tiny: 8q/2kv d64, 4 branches, prefix 256 + suffix 32",
