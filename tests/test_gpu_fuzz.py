@@ -57,3 +57,37 @@ def test_random_segment_structures_match_the_oracle(first):
             check_attention(out.cpu().numpy(), rk.split_block_mass(plan, mass), ref_out, ref_m)
         except AssertionError as e:
             raise AssertionError(f"seed {seed}: {e}") from None
+
+
+def test_random_gate_shapes_match_the_oracle():
+    """The gate over random shapes (1-69 branches, 1-8 roots, 1-40 layers, hidden sizes from 1 to 4097
+    including ones that are no multiple of four), random perturbation levels, alpha and tau from the
+    paper's grids, now and then a zero-norm layer vector: map bit-exact wherever the oracle's sigma
+    keeps 1e-3 clear of tau, sigma within 2e-5."""
+    import torch
+    import oracle
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+    checked = 0
+    for trial in range(90):
+        rng = np.random.default_rng(trial)
+        B, P, L = int(rng.integers(1, 70)), int(rng.integers(1, 9)), int(rng.integers(1, 41))
+        D = int(rng.choice([1, 3, 4, 7, 64, 100, 255, 256, 1000, 1024, 3584, 4096, 4097]))
+        cand = rng.integers(0, P, size=B).astype(np.int32)
+        eps = [float(rng.choice([0.0, 0.1, 0.203, 0.5, 0.75, 1.5, np.inf])) for _ in range(B)]
+        alpha = float(rng.choice([0.0, 0.5, 1.0, 1.5, 2.0]))
+        tau = float(rng.choice([0.0, 0.5, 0.82, 0.9, 0.95]))
+        g = workloads.make_gate_inputs(cand, P, L, D, eps, alpha=alpha, tau=tau, seed=trial)
+        hb = g.h_branch.clone()
+        if trial % 9 == 0:
+            hb[0, 0] = 0.0
+        m_ref, s_ref = oracle.asks_gate(hb.numpy(), g.h_root.numpy(), cand, alpha, tau)
+        if np.abs(s_ref - np.float32(tau)).min() < 1e-3:
+            continue
+        m, s = rk.rksc_asks_gate(hb.to(dev), g.h_root.to(dev), torch.from_numpy(cand).to(dev), alpha, tau)
+        torch.cuda.synchronize()
+        assert np.array_equal(m.cpu().numpy(), m_ref), trial
+        assert np.abs(s.cpu().numpy() - s_ref).max() <= 2e-5, trial
+        checked += 1
+    assert checked >= 60
