@@ -91,3 +91,46 @@ def test_random_gate_shapes_match_the_oracle():
         assert np.abs(s.cpu().numpy() - s_ref).max() <= 2e-5, trial
         checked += 1
     assert checked >= 60
+
+
+def test_random_eviction_problems_match_algorithm_4():
+    """RSBCM selection on random scores and depths (sizes around the kernel's 32 / 256 / 1024 boundaries,
+    capacities from 0 to more than n, with and without ties) against the oracle that evicts the arg-min
+    one entry at a time: the same entries, bit for bit."""
+    import torch
+    import oracle
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+    for trial in range(70):
+        rng = np.random.default_rng(trial)
+        n = int(rng.choice([1, 2, 7, 31, 32, 33, 255, 256, 257, 700, 1023, 1024, 1025]))
+        cap = int(rng.integers(0, n + 2))
+        score, depth = workloads.make_eviction_inputs(n, seed=trial, tie_levels=int(rng.choice([0, 0, 2, 5, 50])))
+        ref = oracle.rsbcm_evict(score, depth, cap)[0]
+        ev, cnt = rk.rksc_rsbcm_evict(torch.from_numpy(score).to(dev), torch.from_numpy(depth).to(dev), cap)
+        torch.cuda.synchronize()
+        assert np.array_equal(ev.cpu().numpy().astype(bool), ref), (trial, n, cap)
+        assert int(cnt.item()) == int(ref.sum()), (trial, n, cap)
+
+
+def test_random_unembedding_shapes_match_the_entropy_oracle():
+    """Entropy and top-1 probability of softmax(h W_u^T) over random shapes (1-32 rows, vocabularies from
+    1 to 50257 entries around the 128-row tile, flat and peaked logits)."""
+    import torch
+    import oracle
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+    for trial in range(20):
+        rng = np.random.default_rng(100 + trial)
+        B = int(rng.integers(1, 33))
+        D = int(rng.choice([64, 128, 512, 1000, 3584]))
+        V = int(rng.choice([1, 5, 127, 128, 129, 1000, 32000, 50257]))
+        h, w = workloads.make_cgee_inputs(B, D, V, seed=trial, logit_std=float(rng.choice([0.5, 3.0, 8.0])))
+        H_ref, p_ref = oracle.logit_entropy(oracle.to_f32_numpy(h), oracle.to_f32_numpy(w))
+        H, p, status = rk.rksc_cgee_logit_entropy(h.to(dev), w.to(dev))[:3]
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, trial
+        assert np.abs(H.cpu().numpy() - H_ref).max() <= 2e-3, (trial, B, D, V)
+        assert (np.abs(p.cpu().numpy() - p_ref) / p_ref).max() <= 2e-3, (trial, B, D, V)
