@@ -134,3 +134,31 @@ def test_random_unembedding_shapes_match_the_entropy_oracle():
         assert int(status.item()) == 0, trial
         assert np.abs(H.cpu().numpy() - H_ref).max() <= 2e-3, (trial, B, D, V)
         assert (np.abs(p.cpu().numpy() - p_ref) / p_ref).max() <= 2e-3, (trial, B, D, V)
+
+
+def test_random_suffix_prefill_problems_match_the_oracle():
+    """Suffix prefill (s in 1..16 query tokens per branch, causal inside the suffix) over random shared /
+    private segment structures whose last segment holds s tokens or a few more: the library's
+    virtual-branch tables bit-exact against the oracle's, outputs and masses within the tolerances."""
+    from test_gpu_suffix_prefill import _run
+
+    edge = [1, 2, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129]
+    for seed in range(60):
+        rng = np.random.default_rng(seed)
+        s = int(rng.choice([1, 2, 3, 5, 8, 16]))
+        hd, Hkv, G = int(rng.choice([64, 128, 128])), int(rng.choice([1, 2, 4])), int(rng.choice([1, 4, 7]))
+        B = int(rng.integers(1, 12))
+        seg_ntok, br = [], [[] for _ in range(B)]
+        for sh in range(int(rng.integers(0, 3))):
+            seg_ntok.append(int(rng.choice(edge)) if rng.random() < 0.5 else int(rng.integers(1, 400)))
+            for b in rng.choice(B, size=int(rng.integers(1, B + 1)), replace=False):
+                br[int(b)].append(sh)
+        for b in range(B):
+            extra = int(rng.choice([0, 1, 15, 16, 17])) if rng.random() < 0.6 else int(rng.integers(0, 120))
+            seg_ntok.append(s + extra)
+            br[b] = sorted(br[b]) + [len(seg_ntok) - 1]
+        w = workloads.make_from_segments(f"pf{seed}", Hkv * G, Hkv, hd, seg_ntok, br, seed=3000 + seed)
+        try:
+            _run(w, s, seed=seed)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed} (s = {s}): {e}") from None
