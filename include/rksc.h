@@ -195,7 +195,9 @@ RKSC_API void    rksc_plan_destroy(rksc_plan* plan);
  *            it after synchronising.
  * Each prefix page shared by n branches is fetched from HBM once per KV head and serves all
  * n * (Hq/Hkv) stacked query rows.  A branch without tokens gets out = 0.
- * Launches: one segment-attention kernel + one merge kernel on `stream`.
+ * Launches: the segment-attention kernels (tensor-core and / or warp-MMA, as the plan needs) and one
+ * merge kernel on `stream`.  Work is handed out dynamically, but every work item's arithmetic and the
+ * order of the merge are fixed: the same plan and inputs give the same bits on every call.
  * ------------------------------------------------------------------------------------------ */
 RKSC_API int32_t rksc_branch_decode_attention(const rksc_plan* plan, const void* q,
                                      const void* k_pool, const void* v_pool,
