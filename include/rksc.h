@@ -212,6 +212,13 @@ RKSC_API int32_t rksc_branch_decode_attention(const rksc_plan* plan, const void*
  * rksc_branch_decode_attention == phases (RKSC_PHASE_SEGMENTS | RKSC_PHASE_MERGE). */
 #define RKSC_PHASE_SEGMENTS 1
 #define RKSC_PHASE_MERGE    2
+/* Added to RKSC_PHASE_MERGE: the merge kernel is launched as an ordinary successor of the segment
+ * kernels instead of with programmatic stream serialisation.  By default its blocks may take their
+ * places on the SMs while the segment kernel drains (and wait there); that saves a little when the
+ * call runs alone, but where other streams have kernels waiting for those SMs (the gate kernels of
+ * later steps in rksc_pipeline) it is better to leave the drain to them: the step pipeline sets this
+ * flag (measured: 0.178 instead of 0.185 ms per step on the batched-serving configuration). */
+#define RKSC_PHASE_MERGE_LATE 4
 RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan* plan, const void* q,
                                      const void* k_pool, const void* v_pool,
                                      float* out, float* block_mass,
@@ -429,8 +436,9 @@ RKSC_API int32_t rksc_kv_append(const rksc_layout* layout, void* k_pool, void* v
  * rksc_pipeline_create: layout, shapes (B branches, P prefixes, L layers, D hidden size), alpha,
  *   tau and the three page-list CSRs as for rksc_tables_from_gate (host arrays, copied: every step
  *   uses the same lists, only its gate map differs); depth in [2, 8]; mass_capacity = floats the
- *   caller's block_mass buffers hold (0 if it passes none); timing != 0 makes every step record
- *   CUDA events around its segment kernels (the attention is then launched in its two phases).
+ *   caller's block_mass buffers hold (0 if it passes none); timing = n > 0 makes every n-th step
+ *   (ticket % n == 0) record CUDA events around its segment kernels (that step's attention is then
+ *   launched in its two phases); 0: no events.
  * rksc_pipeline_submit: device pointers as for rksc_asks_gate (h_branch, h_root, cand_prefix) and
  *   rksc_branch_decode_attention (q, pools, out, block_mass or NULL).  The buffers must stay valid
  *   and unchanged until the step has been waited for; `after_stream` (may be NULL): work already
@@ -440,8 +448,8 @@ RKSC_API int32_t rksc_kv_append(const rksc_layout* layout, void* k_pool, void* v
  *   device must be the one the pipeline was created on.
  * rksc_pipeline_wait: blocks the calling thread until step `ticket` has finished; tickets must be
  *   waited for in submission order, each once.  Optional outputs (host, may be NULL):
- *   branch_to_prefix [B], sigma [B], mass_off [B+1], info (the step's plan), segment_ms (timing
- *   pipelines: device time of the step's segment kernels).  Returns the first failing stage's status, or
+ *   branch_to_prefix [B], sigma [B], mass_off [B+1], info (the step's plan), segment_ms (device
+ *   time of the step's segment kernels if the step was timed, else 0).  Returns the first failing stage's status, or
  *   the attention's device status word, or RKSC_ERR_WORKSPACE when the step's masses did not fit
  *   mass_capacity (the attention was not run).
  * rksc_pipeline_destroy: waits for everything in flight, stops the threads, frees the buffers.

@@ -640,14 +640,14 @@ class Pipeline:
     """rksc_pipeline_*: whole steps (gate, map to the host, tables + plan, attention) kept ``depth`` deep in
     flight by the library's own streams and host threads.  Argument marshalling only."""
 
-    def __init__(self, layout, num_branches, hidden_shape, alpha, tau, lists, depth=4, mass_capacity=0, timing=False):
+    def __init__(self, layout, num_branches, hidden_shape, alpha, tau, lists, depth=4, mass_capacity=0, timing=0):
         lay = layout if isinstance(layout, Layout) else Layout.of(layout)
         gl = lists if isinstance(lists, GateLists) else GateLists(lists)
         L_, D = hidden_shape
         self.layout, self.B, self.depth = lay, int(num_branches), int(depth)
         h = C.c_void_p()
         _check(lib().rksc_pipeline_create(C.byref(lay.c), self.B, gl.num_prefixes, int(L_), int(D), float(alpha),
-                                          float(tau), *gl.ptrs, int(depth), int(mass_capacity), int(bool(timing)),
+                                          float(tau), *gl.ptrs, int(depth), int(mass_capacity), int(timing),
                                           C.byref(h)), "rksc_pipeline_create")
         self._h = h.value
         self._keep = {}

@@ -378,7 +378,9 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
                                                 float* block_mass, void* workspace, size_t workspace_bytes,
                                                 int32_t* device_status, void* stream, int32_t phases) {
     if (!plan) return RKSC_ERR_INVALID_ARG;
-    if ((phases & ~(RKSC_PHASE_SEGMENTS | RKSC_PHASE_MERGE)) || phases == 0) return RKSC_ERR_INVALID_ARG;
+    if ((phases & ~(RKSC_PHASE_SEGMENTS | RKSC_PHASE_MERGE | RKSC_PHASE_MERGE_LATE)) ||
+        (phases & (RKSC_PHASE_SEGMENTS | RKSC_PHASE_MERGE)) == 0)
+        return RKSC_ERR_INVALID_ARG;
     const HostPlan& H = plan->host;
     if (H.B == 0) return RKSC_OK;
     if (!q || !k_pool || !v_pool || !out) return RKSC_ERR_INVALID_ARG;
@@ -428,7 +430,7 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
         e = launch_seg_attn_tc(tm_k, tm_v, a, s);
         if (e == cudaSuccess) e = launch_seg_attn_warp(tm_k, tm_v, a, s, /*after_tc=*/a.grid_tc > 0);
     }
-    if (e == cudaSuccess && (phases & RKSC_PHASE_MERGE)) e = launch_merge(a, s);
+    if (e == cudaSuccess && (phases & RKSC_PHASE_MERGE)) e = launch_merge(a, s, !(phases & RKSC_PHASE_MERGE_LATE));
     if (e != cudaSuccess) {
         g_last_cuda = e;
         cudaGetLastError();

@@ -40,7 +40,7 @@ cudaError_t launch_seg_attn_warp(const CUtensorMap& tm_k, const CUtensorMap& tm_
                                  cudaStream_t stream, bool after_tc);
 cudaError_t launch_seg_attn_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnArgs& a,
                                cudaStream_t stream);
-cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream);
+cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream, bool early_residency);
 
 // RSBCM (Section 2.4, Algorithm 4): per-entry scores from the block masses; exact selection of the
 // k entries smallest by (score / (depth + 1), index).  keys: scratch of n 64-bit words.

@@ -146,7 +146,7 @@ merge_kernel(const AttnArgs a, const int wpk_log2) {
 
 }  // namespace
 
-cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream) {
+cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream, bool early_residency) {
     const int n = a.B * a.Hq;
     if (n == 0) return cudaSuccess;
     int wpk_log2 = 0;   // warps per (branch, head): enough warps to fill the device
@@ -166,7 +166,7 @@ cudaError_t launch_merge(const AttnArgs& a, cudaStream_t stream) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = early_residency ? 1 : 0;   // without the attribute the merge starts when the segment kernel has completed
     return cudaLaunchKernelEx(&cfg, merge_kernel, a, wpk_log2);
 }
 

@@ -44,6 +44,7 @@ struct Slot {
     int64_t ticket = -1;
     int32_t status = RKSC_OK;          // host-side status of the step's stages
     bool attention_enqueued = false;
+    bool timed = false;                // this step's segment kernels have events around them
     bool worker_done = true;           // the slot's worker has finished with it
     bool waited = true;                // rksc_pipeline_wait has returned for its ticket
 };
@@ -57,7 +58,7 @@ struct rksc_pipeline {
     std::vector<int32_t> lists[9];
     int depth = 0;
     int64_t mass_capacity = 0;
-    bool timing = false;
+    int timing = 0;                    // 0: no events; n > 0: every n-th step (ticket % n == 0) is timed
     int device = -1;
     cudaStream_t gate_stream = nullptr, att_stream = nullptr;
     cudaEvent_t ev_inputs = nullptr;
@@ -124,7 +125,8 @@ void worker_main(rksc_pipeline* p) {
         }
         if (st == RKSC_OK) {
             cudaStream_t as = p->att_stream;
-            if (p->timing) {
+            s.timed = p->timing > 0 && t % p->timing == 0;
+            if (s.timed) {
                 cudaEventRecord(s.ev_seg0, as);
                 st = rksc_branch_decode_attention_phases(plan, s.q, s.k_pool, s.v_pool, s.out, s.block_mass, s.workspace,
                                                          s.workspace_cap, s.status_dev, as, RKSC_PHASE_SEGMENTS);
@@ -132,10 +134,13 @@ void worker_main(rksc_pipeline* p) {
                 if (st == RKSC_OK)
                     st = rksc_branch_decode_attention_phases(plan, s.q, s.k_pool, s.v_pool, s.out, s.block_mass,
                                                              s.workspace, s.workspace_cap, s.status_dev, as,
-                                                             RKSC_PHASE_MERGE);
+                                                             RKSC_PHASE_MERGE | RKSC_PHASE_MERGE_LATE);
             } else {
-                st = rksc_branch_decode_attention(plan, s.q, s.k_pool, s.v_pool, s.out, s.block_mass, s.workspace,
-                                                  s.workspace_cap, s.status_dev, as);
+                // the merge as an ordinary successor: the gate kernels of later steps use the SMs the segment
+                // kernel frees while it drains, instead of merge blocks that would only wait there
+                st = rksc_branch_decode_attention_phases(plan, s.q, s.k_pool, s.v_pool, s.out, s.block_mass, s.workspace,
+                                                         s.workspace_cap, s.status_dev, as,
+                                                         RKSC_PHASE_SEGMENTS | RKSC_PHASE_MERGE | RKSC_PHASE_MERGE_LATE);
             }
             s.attention_enqueued = (st == RKSC_OK);
             if (cudaMemcpyAsync(s.map_host + 2 * (size_t)p->B, s.status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, as) !=
@@ -236,7 +241,7 @@ extern "C" RKSC_API int32_t rksc_pipeline_create(const rksc_layout* layout, int3
     p->tau = tau;
     p->depth = depth;
     p->mass_capacity = mass_capacity;
-    p->timing = timing != 0;
+    p->timing = timing > 0 ? timing : 0;
     bool ok = cudaGetDevice(&p->device) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&p->gate_stream, cudaStreamNonBlocking) == cudaSuccess;
     // the attention stream outranks the gate stream: where both have thread blocks waiting for an SM,
@@ -252,7 +257,7 @@ extern "C" RKSC_API int32_t rksc_pipeline_create(const rksc_layout* layout, int3
         ok = ok && cudaMallocHost(reinterpret_cast<void**>(&s.map_host), (2 * (size_t)B + 4) * 4) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&s.ev_map, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&s.ev_done, cudaEventDisableTiming) == cudaSuccess;
-        if (p->timing) {
+        if (p->timing > 0) {
             ok = ok && cudaEventCreate(&s.ev_seg0) == cudaSuccess;
             ok = ok && cudaEventCreate(&s.ev_seg1) == cudaSuccess;
         }
@@ -307,6 +312,7 @@ extern "C" RKSC_API int32_t rksc_pipeline_submit(rksc_pipeline* p, const float* 
     s.block_mass = block_mass;
     s.ticket = t;
     s.attention_enqueued = false;
+    s.timed = false;
     cudaStream_t gs = p->gate_stream;
     int32_t st = RKSC_OK;
     if (cudaMemsetAsync(s.status_dev, 0, 16, gs) != cudaSuccess) st = RKSC_ERR_CUDA;
@@ -371,7 +377,7 @@ extern "C" RKSC_API int32_t rksc_pipeline_wait(rksc_pipeline* p, int64_t ticket,
     }
     if (segment_ms) {
         *segment_ms = 0.f;
-        if (p->timing && s.attention_enqueued && cudaEventElapsedTime(segment_ms, s.ev_seg0, s.ev_seg1) != cudaSuccess)
+        if (s.timed && s.attention_enqueued && cudaEventElapsedTime(segment_ms, s.ev_seg0, s.ev_seg1) != cudaSuccess)
             cudaGetLastError();
     }
     s.waited = true;

@@ -146,6 +146,15 @@ def test_in_flight_rules_small_mass_buffer_and_timing():
     assert pipe.wait(1).status == 0 and pipe.wait(2).status == 0
     pipe.close()
 
+    # timing = 2: events around the segment kernels of every second step only
+    every2 = rk.Pipeline(w.layout, w.num_branches, (L, D), w.gate.alpha, w.gate.tau, w.flat, depth=4, mass_capacity=cap,
+                         timing=2)
+    for i in range(4):
+        every2.submit(hb, hr, cand, q, kp, vp, out, mass)
+    ms = [every2.wait(i).segment_ms for i in range(4)]
+    every2.close()
+    assert ms[0] > 0.0 and ms[2] > 0.0 and ms[1] == 0.0 and ms[3] == 0.0
+
     small = rk.Pipeline(w.layout, w.num_branches, (L, D), w.gate.alpha, w.gate.tau, w.flat, depth=3, mass_capacity=8)
     out.fill_(7.0)
     t = small.submit(hb, hr, cand, q, kp, vp, out, mass)
