@@ -266,3 +266,23 @@ def test_long_prefix_serving_sampled():
     sample = sorted(set(rng.choice(priv, 3, replace=False).tolist() + rng.choice(shared, 5, replace=False).tolist()))
     ref_out, ref_m = oracle_attention(w, t, branches=sample)
     check_attention(out, m, ref_out, ref_m, branches=sample)
+
+
+def test_late_merge_gives_the_same_bits_and_bad_phase_words_are_refused():
+    """RKSC_PHASE_MERGE_LATE only changes how the merge kernel is launched (an ordinary successor instead
+    of programmatic serialisation), not what it computes."""
+    import torch
+    import paper_2606_09937_b200 as rk
+
+    dev = torch.device("cuda:0")
+    w = workloads.make_config("qwen_layer")
+    t = oracle_tables_from_map(w, oracle_gate(w.gate)[0])
+    plan = rk.rksc_plan_create(w.layout, t)
+    q, kp, vp = w.q.to(dev), w.k_pool.to(dev), w.v_pool.to(dev)
+    out0, mass0, _ = rk.rksc_branch_decode_attention(plan, q, kp, vp)
+    out1, mass1, st = rk.rksc_branch_decode_attention(plan, q, kp, vp, phases=1 | 2 | 4)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and torch.equal(out0, out1) and torch.equal(mass0, mass1)
+    for bad in (0, 4, 8, 16 | 1):
+        with pytest.raises(rk.RkscError):
+            rk.rksc_branch_decode_attention(plan, q, kp, vp, phases=bad)
