@@ -177,8 +177,16 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
             int want = std::min(cap, std::max(base, 2 * rows));
             if (klass == 1) want = tc_chunk;
             const int nch = ceil_div(np, want);
+            // chunk c covers pages [np * c / nch, np * (c + 1) / nch): one division per chunk, in 32 bits
+            // where the product fits (64-bit divisions were a third of this loop's time)
+            const bool narrow = (int64_t)np * nch < ((int64_t)1 << 31);
+            auto cut = [&](int c) {
+                return narrow ? (int)((uint32_t)np * (uint32_t)c / (uint32_t)nch) : (int)((int64_t)np * c / nch);
+            };
+            int p_hi = 0;
             for (int c = 0; c < nch; ++c) {
-                const int p_lo = (int)((int64_t)np * c / nch), p_hi = (int)((int64_t)np * (c + 1) / nch);
+                const int p_lo = p_hi;
+                p_hi = cut(c + 1);
                 const int tok_lo = p_lo * kBlock;
                 const int tok_hi = std::min(P.seg_num_tokens[s], p_hi * kBlock);
                 for (int h = 0; h < L.num_kv_heads; ++h) {
