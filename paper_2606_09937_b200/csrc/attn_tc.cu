@@ -1,5 +1,5 @@
 // Segment attention on the 5th-generation tensor cores (tcgen05 + TMEM) for work items with
-// 17..128 stacked query rows and head_dim 128.
+// 9..128 stacked query rows and head_dim 128.
 //
 // All branches that share a segment, times the G query heads of a KV head, are stacked into the
 // 128 rows of one MMA tile; a KV page staged in shared memory once then serves every sharing

@@ -11,7 +11,7 @@ namespace rksc {
 
 constexpr int kBlock = RKSC_BLOCK_SIZE;     // tokens per KV page
 constexpr int kMaxRowsPerItem = 64;         // stacked query rows one warp-MMA work item handles
-constexpr int kTcMinRows = 17;              // from this many stacked rows on, the tcgen05 kernel takes the item
+constexpr int kTcMinRows = 9;               // from this many stacked rows on, the tcgen05 kernel takes the item (up to 8: the warp kernel's transposed small-row path)
 constexpr int kTcMaxRows = 128;             // rows of one tcgen05 work item (the MMA's M)
 constexpr int kMaxPagesPerItem = 512;       // page ids a CTA caches in shared memory
 constexpr int kConsumerWarps = 4;           // MMA warps of the segment kernel
