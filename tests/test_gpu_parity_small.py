@@ -48,9 +48,11 @@ def test_ragged_segments(hq, hkv, d):
     _parity(w)
 
 
-@pytest.mark.parametrize("sharers,G", [(1, 1), (3, 5), (9, 7), (16, 4), (17, 4), (4, 16), (33, 2), (70, 1)])
+@pytest.mark.parametrize("sharers,G", [(1, 1), (2, 4), (8, 1), (9, 1), (3, 3), (3, 4), (3, 5), (2, 8), (9, 7), (16, 4),
+                                       (17, 4), (4, 16), (33, 2), (70, 1)])
 def test_row_counts_around_tile_edges(sharers, G):
-    # stacked rows = sharers * G: 1, 15, 63, 64, 68 (two sharer blocks), 64, 66, 70
+    # stacked rows = sharers * G: 1, 8, 8 (the last counts of the warp kernel's small-row path), 9, 9, 12, 15,
+    # 16 (the first counts of the tcgen05 kernel), 63, 64, 68 (two sharer blocks), 64, 66, 70
     hkv = 2
     w = workloads.make_from_segments("rows", G * hkv, hkv, 128, [200] + [19] * sharers,
                                      [[0, 1 + b] for b in range(sharers)], seed=12 + sharers)
