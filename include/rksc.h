@@ -427,7 +427,7 @@ RKSC_API int32_t rksc_kv_append(const rksc_layout* layout, void* k_pool, void* v
  *
  * The tables of a step depend on its gate map, which has to come to the host; a caller that runs
  * the four stages one after another leaves the GPU idle while the host builds the plan.  The
- * pipeline owns two streams and depth - 2 (at least one) host threads: rksc_pipeline_submit
+ * pipeline owns its streams (gate, attention, status copies) and depth - 2 (at least one) host threads: rksc_pipeline_submit
  * enqueues the step's gate kernel and the copy of its map on the gate stream and returns; a host
  * thread waits for that copy, builds tables and plan, and enqueues the attention on the attention
  * stream - in submission order, so that attention launches run back to back while the gates of

@@ -38,6 +38,7 @@ struct Slot {
     void* workspace = nullptr;
     size_t workspace_cap = 0;
     cudaEvent_t ev_map = nullptr;      // gate + map copy done
+    cudaEvent_t ev_att = nullptr;      // attention enqueued on the attention stream is done
     cudaEvent_t ev_done = nullptr;     // attention + status copy done
     cudaEvent_t ev_seg0 = nullptr, ev_seg1 = nullptr;   // timing pipelines
     rksc_plan* plan = nullptr;
@@ -61,6 +62,7 @@ struct rksc_pipeline {
     int timing = 0;                    // 0: no events; n > 0: every n-th step (ticket % n == 0) is timed
     int device = -1;
     cudaStream_t gate_stream = nullptr, att_stream = nullptr;
+    cudaStream_t copy_stream = nullptr;   // status words back to the host, off the attention stream
     cudaEvent_t ev_inputs = nullptr;
     std::vector<Slot> slots;
     int64_t next_ticket = 0;           // submitting thread only
@@ -143,9 +145,13 @@ void worker_main(rksc_pipeline* p) {
                                                          RKSC_PHASE_SEGMENTS | RKSC_PHASE_MERGE | RKSC_PHASE_MERGE_LATE);
             }
             s.attention_enqueued = (st == RKSC_OK);
-            if (cudaMemcpyAsync(s.map_host + 2 * (size_t)p->B, s.status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, as) !=
+            // The status word goes back on a stream of its own, behind an event: a copy between two steps'
+            // kernels on the attention stream would put a copy-engine round trip between them.
+            cudaStream_t cs = p->copy_stream;
+            if (cudaEventRecord(s.ev_att, as) != cudaSuccess || cudaStreamWaitEvent(cs, s.ev_att, 0) != cudaSuccess ||
+                cudaMemcpyAsync(s.map_host + 2 * (size_t)p->B, s.status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, cs) !=
                     cudaSuccess ||
-                cudaEventRecord(s.ev_done, as) != cudaSuccess) {
+                cudaEventRecord(s.ev_done, cs) != cudaSuccess) {
                 cudaGetLastError();
                 if (st == RKSC_OK) st = RKSC_ERR_CUDA;
             }
@@ -169,7 +175,7 @@ void free_slot(Slot& s) {
     if (s.status_dev) cudaFree(s.status_dev);
     if (s.map_host) cudaFreeHost(s.map_host);
     if (s.workspace) cudaFree(s.workspace);
-    for (cudaEvent_t e : {s.ev_map, s.ev_done, s.ev_seg0, s.ev_seg1})
+    for (cudaEvent_t e : {s.ev_map, s.ev_att, s.ev_done, s.ev_seg0, s.ev_seg1})
         if (e) cudaEventDestroy(e);
     s = Slot{};
 }
@@ -190,10 +196,12 @@ extern "C" RKSC_API void rksc_pipeline_destroy(rksc_pipeline* p) {
         if (w.joinable()) w.join();   // workers finish the queued steps first
     if (p->gate_stream) cudaStreamSynchronize(p->gate_stream);
     if (p->att_stream) cudaStreamSynchronize(p->att_stream);
+    if (p->copy_stream) cudaStreamSynchronize(p->copy_stream);
     for (auto& s : p->slots) free_slot(s);
     if (p->ev_inputs) cudaEventDestroy(p->ev_inputs);
     if (p->gate_stream) cudaStreamDestroy(p->gate_stream);
     if (p->att_stream) cudaStreamDestroy(p->att_stream);
+    if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
     cudaGetLastError();
     if (sw) cudaSetDevice(cur);
     delete p;
@@ -249,6 +257,7 @@ extern "C" RKSC_API int32_t rksc_pipeline_create(const rksc_layout* layout, int3
     int prio_lo = 0, prio_hi = 0;
     ok = ok && cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess;
     ok = ok && cudaStreamCreateWithPriority(&p->att_stream, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&p->ev_inputs, cudaEventDisableTiming) == cudaSuccess;
     for (auto& s : p->slots) {
         ok = ok && cudaMalloc(reinterpret_cast<void**>(&s.map_dev), (size_t)B * 4) == cudaSuccess;
@@ -256,6 +265,7 @@ extern "C" RKSC_API int32_t rksc_pipeline_create(const rksc_layout* layout, int3
         ok = ok && cudaMalloc(reinterpret_cast<void**>(&s.status_dev), 16) == cudaSuccess;
         ok = ok && cudaMallocHost(reinterpret_cast<void**>(&s.map_host), (2 * (size_t)B + 4) * 4) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&s.ev_map, cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&s.ev_att, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&s.ev_done, cudaEventDisableTiming) == cudaSuccess;
         if (p->timing > 0) {
             ok = ok && cudaEventCreate(&s.ev_seg0) == cudaSuccess;
