@@ -318,22 +318,22 @@ extern "C" RKSC_API int32_t rksc_plan_query(const rksc_plan* plan, rksc_plan_inf
     info->workspace_bytes = H.workspace_bytes;
     info->mass_elems = H.mass_elems;
     info->mass_off = H.mass_off.data();
-    info->num_work_items = (int32_t)H.items.size();
+    info->num_work_items = H.num_work_items;
     info->num_partial_rows = H.num_partial_rows;
     info->unique_kv_tokens = H.unique_kv_tokens;
     info->duplicated_kv_tokens = H.duplicated_kv_tokens;
     info->on_device = plan->on_device ? 1 : 0;
     info->num_pages_listed = (int64_t)H.seg_blocks.size();
     info->num_kernel_launches = H.B == 0 ? 0 : (H.num_tc_items > 0 ? 1 : 0) +
-                                                   ((int)H.items.size() > H.num_tc_items ? 1 : 0) + 1;
+                                                   (H.num_work_items > H.num_tc_items ? 1 : 0) + 1;
     return RKSC_OK;
 }
 
 extern "C" RKSC_API int32_t rksc_plan_get_item(const rksc_plan* plan, int32_t i, int32_t* out10) {
     if (!plan || !out10) return RKSC_ERR_INVALID_ARG;
     const HostPlan& H = plan->host;
-    if (i < 0 || i >= (int32_t)H.items.size()) return RKSC_ERR_INVALID_ARG;
-    const WorkItem& it = H.items[i];
+    if (i < 0 || i >= H.num_work_items) return RKSC_ERR_INVALID_ARG;
+    const WorkItem it = work_item_of(H.items.data(), i, H.layout.num_kv_heads, H.G);
     out10[0] = it.seg;
     out10[1] = it.kv_head;
     out10[2] = it.seg_page_begin;
@@ -410,7 +410,7 @@ extern "C" RKSC_API int32_t rksc_branch_decode_attention_phases(const rksc_plan*
     a.out = out;
     a.status = device_status;
     a.counters = plan->dev.counters;
-    a.num_items = (int)H.items.size();
+    a.num_items = H.num_work_items;
     a.num_tc_items = H.num_tc_items;
     a.grid_warp = H.grid_warp;
     a.grid_tc = H.grid_tc;

@@ -293,7 +293,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     // anything else, so that the round trip passes behind the set-up below (the plan's arrays are
     // written by no kernel: reading them does not have to wait for the kernel before this one).
     WorkItem it_first{};
-    if ((warp == kProducerWarp || warp == kQWarp) && (int)blockIdx.x < a.num_tc_items) it_first = a.plan.items[blockIdx.x];
+    if ((warp == kProducerWarp || warp == kQWarp) && (int)blockIdx.x < a.num_tc_items) it_first = work_item_of(a.plan.items, blockIdx.x, a.Hkv, a.G);
     if (tid == 0) {
         for (int i = 0; i < kNK; ++i) {
             mbar_init(bar(kBarFullK + i), 1);
@@ -370,7 +370,7 @@ seg_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         };
         auto fetch_item = [&](int i) {
             WorkItem w{};
-            if (i < a.num_tc_items) w = a.plan.items[i];
+            if (i < a.num_tc_items) w = work_item_of(a.plan.items, i, a.Hkv, a.G);
             return w;
         };
         auto fetch_ids = [&](const WorkItem& w, int first) {

@@ -263,7 +263,7 @@ seg_attn_warp_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         };
         auto fetch_item = [&](int i) {
             WorkItem w{};
-            if (i < a.num_items) w = a.plan.items[i];
+            if (i < a.num_items) w = work_item_of(a.plan.items, i, a.Hkv, a.G);
             return w;
         };
         auto fetch_ids = [&](const WorkItem& w, int first) {   // page ids first + lane of the item (0 past its end)

@@ -148,22 +148,17 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
     // neutral on the other configurations.
     const int tc_chunk = (int)std::min<int64_t>(kMaxPagesPerItem, std::max<int64_t>(kMinChunk, fair * 2));
     int64_t rows_total = 0;
-    {
-        size_t n_items = 0;   // exact count, so that the item vector is allocated once
-        for (int s = 0; s < S; ++s) {
-            const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
-            const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
-            if (ns == 0 || np == 0) continue;
-            const int nsb = ceil_div(ns, seg_rows_per_block(ns));
-            for (int sb = 0; sb < nsb; ++sb) {
-                const int rows = ((int)((int64_t)ns * (sb + 1) / nsb) - (int)((int64_t)ns * sb / nsb)) * G;
-                int want0 = std::min(cap, std::max(base, 2 * rows));
-                if (tc_ok && rows >= kTcMinRows) want0 = tc_chunk;
-                n_items += (size_t)ceil_div(np, want0) * L.num_kv_heads;
-            }
-        }
-        P.items.reserve(n_items);
-    }
+    // Items are created in segment order and handed to the kernels sorted by (class, cost / 16), long
+    // items first; the bucket of every item and the bucket counts are taken while the items are made,
+    // so that the sort below is one scatter.  (A plan object is recycled with its vectors' capacity:
+    // nothing is counted ahead.)
+    constexpr int kBuckets = 1024;
+    std::vector<int32_t>& bucket_of = P.scratch_a;
+    bucket_of.clear();
+    int32_t count[2][kBuckets + 1];
+    std::memset(count, 0, sizeof(count));
+    std::vector<WorkItem>& made = P.scratch_items;
+    made.clear();
     for (int s = 0; s < S; ++s) {
         const int ns = P.seg_sharer_off[s + 1] - P.seg_sharer_off[s];
         const int np = P.seg_block_off[s + 1] - P.seg_block_off[s];
@@ -189,43 +184,34 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
                 p_hi = cut(c + 1);
                 const int tok_lo = p_lo * kBlock;
                 const int tok_hi = std::min(P.seg_num_tokens[s], p_hi * kBlock);
-                for (int h = 0; h < L.num_kv_heads; ++h) {
-                    WorkItem it{};
-                    it.seg = s;
-                    it.kv_head = h;
-                    it.page_begin = P.seg_block_off[s] + p_lo;
-                    it.num_pages = p_hi - p_lo;
-                    it.num_tokens = tok_hi - tok_lo;
-                    it.sharer_begin = P.seg_sharer_off[s] + sh_lo;
-                    it.num_sharers = sh_hi - sh_lo;
-                    it.part_row_base = 0;  // set after sorting
-                    it.seg_page_begin = p_lo;
-                    it.klass = klass;
-                    P.items.push_back(it);
-                    rows_total += rows;
-                }
+                WorkItem it{};
+                it.seg = s;
+                it.page_begin = P.seg_block_off[s] + p_lo;
+                it.num_pages = p_hi - p_lo;
+                it.num_tokens = tok_hi - tok_lo;
+                it.sharer_begin = P.seg_sharer_off[s] + sh_lo;
+                it.num_sharers = sh_hi - sh_lo;
+                it.part_row_base = 0;  // set after sorting
+                it.seg_page_begin = p_lo;
+                it.klass = klass;
+                const int64_t cost = item_cost(it, G);
+                const int bkt = kBuckets - 1 - (int)std::min<int64_t>(kBuckets - 1, cost >> 4);   // small index = long item
+                count[1 - klass][bkt + 1]++;
+                it.kv_head = 0;   // one entry for the chunk's Hkv work items (see WorkItem)
+                made.push_back(it);
+                bucket_of.push_back(bkt);
+                rows_total += (int64_t)rows * L.num_kv_heads;
             }
         }
     }
     if (rows_total >= ((int64_t)1 << 31)) return RKSC_ERR_UNSUPPORTED;
 
     // tensor-core items first, then warp-MMA items; within a class longest first, so that the
-    // CTAs, which claim items in this order, finish together
+    // CTAs, which claim items in this order, finish together.  A counting sort on (class, cost / 16):
+    // descending cost up to the bucket width is all the longest-first claiming needs, it keeps the
+    // order of creation within a bucket, and it is linear in the number of items.
     {
-        // counting sort on (class, cost / 16): descending cost up to the bucket width is all the
-        // longest-first claiming needs, and it is linear in the number of items
-        const size_t n = P.items.size();
-        constexpr int kBuckets = 1024;
-        std::vector<int32_t>& bucket_of = P.scratch_a;
-        bucket_of.resize(n);
-        int32_t count[2][kBuckets + 1];
-        std::memset(count, 0, sizeof(count));
-        for (size_t i = 0; i < n; ++i) {
-            const int64_t cost = item_cost(P.items[i], G);
-            const int bkt = kBuckets - 1 - (int)std::min<int64_t>(kBuckets - 1, cost >> 4);   // small index = long item
-            bucket_of[i] = bkt;
-            count[1 - P.items[i].klass][bkt + 1]++;
-        }
+        const size_t n = made.size();
         int32_t start[2][kBuckets];
         int32_t run = 0;
         for (int c = 0; c < 2; ++c)
@@ -233,38 +219,52 @@ int32_t build_host_plan(const rksc_layout& L, const rksc_tables& t, int num_sms,
                 start[c][b] = run;
                 run += count[c][b + 1];
             }
-        std::vector<WorkItem>& sorted = P.scratch_items;
-        sorted.resize(n);
-        for (size_t i = 0; i < n; ++i) sorted[start[1 - P.items[i].klass][bucket_of[i]]++] = P.items[i];
-        P.items.swap(sorted);
+        P.items.resize(n);
+        for (size_t i = 0; i < n; ++i) P.items[start[1 - made[i].klass][bucket_of[i]]++] = made[i];
     }
     int32_t row = 0;
     P.num_tc_items = 0;
+    const int Hkv = L.num_kv_heads;
+    if ((int64_t)P.items.size() * Hkv >= ((int64_t)1 << 31)) return RKSC_ERR_UNSUPPORTED;
     for (auto& it : P.items) {
         it.part_row_base = row;
-        row += it.num_sharers * G;
-        P.num_tc_items += it.klass;
+        row += it.num_sharers * G * Hkv;
+        P.num_tc_items += it.klass * Hkv;
     }
+    P.num_work_items = (int32_t)P.items.size() * Hkv;
     P.num_partial_rows = row;
     P.grid_tc = std::min(std::max(1, num_sms), P.num_tc_items);
-    P.grid_warp = std::min(max_grid, (int)P.items.size() - P.num_tc_items);
+    P.grid_warp = std::min(max_grid, P.num_work_items - P.num_tc_items);
 
-    // merge lists: for every (branch, kv head) the partial rows (of head-in-group 0) to combine
-    const int nkeys = B * L.num_kv_heads;
-    P.merge_off.assign(nkeys + 1, 0);
-    for (const auto& it : P.items)
-        for (int i = 0; i < it.num_sharers; ++i)
-            P.merge_off[P.sharers[it.sharer_begin + i].branch * L.num_kv_heads + it.kv_head + 1]++;
-    for (int k = 0; k < nkeys; ++k) P.merge_off[k + 1] += P.merge_off[k];
-    P.merge_rows.resize(P.merge_off[nkeys]);
+    // merge lists: for every (branch, kv head) the partial rows (of head-in-group 0) to combine, in item
+    // order.  A branch has the same number of parts under every KV head (an entry of the item array is
+    // Hkv work items), so the parts are counted per branch and laid out head by head.
+    const int nkeys = B * Hkv;
     {
-        std::vector<int32_t>& fill = P.scratch_b;
-        fill.assign(P.merge_off.begin(), P.merge_off.end() - 1);
+        std::vector<int32_t>& cnt = P.scratch_b;   // parts per branch, then the next free position
+        cnt.assign(B, 0);
         for (const auto& it : P.items)
+            for (int i = 0; i < it.num_sharers; ++i) cnt[P.sharers[it.sharer_begin + i].branch]++;
+        P.merge_off.resize(nkeys + 1);
+        int32_t off = 0;
+        for (int b = 0; b < B; ++b) {
+            const int32_t n = cnt[b];
+            for (int h = 0; h < Hkv; ++h) P.merge_off[b * Hkv + h] = off + h * n;
+            off += n * Hkv;
+            cnt[b] = 0;
+        }
+        P.merge_off[nkeys] = off;
+        P.merge_rows.resize(off);
+        for (const auto& it : P.items) {
+            const int R = it.num_sharers * G;
             for (int i = 0; i < it.num_sharers; ++i) {
-                const int key = P.sharers[it.sharer_begin + i].branch * L.num_kv_heads + it.kv_head;
-                P.merge_rows[fill[key]++] = it.part_row_base + i * G;
+                const int b = P.sharers[it.sharer_begin + i].branch;
+                const int pos = cnt[b]++;
+                const int32_t n = P.merge_off[b * Hkv + 1] - P.merge_off[b * Hkv];   // the branch's parts per head
+                for (int h = 0; h < Hkv; ++h)
+                    P.merge_rows[P.merge_off[b * Hkv] + h * n + pos] = it.part_row_base + h * R + i * G;
             }
+        }
     }
 
     // grid of the page-score kernel (RSBCM): 32 consecutive pages of one segment per CTA

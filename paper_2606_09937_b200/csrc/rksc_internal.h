@@ -22,6 +22,9 @@ constexpr int kCtasPerSm = 2;               // persistent CTAs per SM
 
 // One CTA's work: a chunk of one segment's pages for one KV head and a block of the
 // segment's sharers.  Stacked rows = num_sharers * G, row r <-> (sharer r / G, head r % G).
+// The plan's item array holds one entry per (chunk, sharer block) with kv_head = 0; work item i is
+// entry i / Hkv under KV head h = i % Hkv, its partial rows h * num_sharers * G after the entry's
+// (work_item_of below): the Hkv items of a chunk differ in nothing else.
 struct WorkItem {
     int32_t seg;
     int32_t kv_head;
@@ -35,6 +38,18 @@ struct WorkItem {
     int32_t klass;           // 0: warp-MMA kernel, 1: tcgen05 kernel
 };
 static_assert(sizeof(WorkItem) == 40, "WorkItem is read as 10 int32");
+
+// Work item i of a plan whose item array is `entries` (host and device).
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline WorkItem work_item_of(const WorkItem* entries, int i, int Hkv, int G) {
+    const int e = i / Hkv, h = i - e * Hkv;
+    WorkItem w = entries[e];
+    w.kv_head = h;
+    w.part_row_base += h * w.num_sharers * G;
+    return w;
+}
 
 // A (segment, branch) incidence: where the branch's masses of this segment start.
 struct Sharer {
@@ -64,7 +79,8 @@ struct HostPlan {
     std::vector<int32_t> seg_block_off;
     std::vector<int32_t> seg_num_tokens;
     std::vector<WorkItem> items;
-    int32_t num_tc_items = 0;             // items [0, num_tc_items) belong to the tcgen05 kernel
+    int32_t num_work_items = 0;           // items.size() * Hkv
+    int32_t num_tc_items = 0;             // work items [0, num_tc_items) belong to the tcgen05 kernel
     int32_t grid_tc = 0, grid_warp = 0;   // persistent CTAs of the two segment kernels
     std::vector<Sharer> sharers;
     std::vector<int32_t> seg_sharer_off;  // [S+1]
@@ -91,7 +107,7 @@ struct HostPlan {
         seg_block_off.clear();
         seg_num_tokens.clear();
         items.clear();
-        num_tc_items = grid_tc = grid_warp = 0;
+        num_work_items = num_tc_items = grid_tc = grid_warp = 0;
         sharers.clear();
         seg_sharer_off.clear();
         merge_off.clear();
