@@ -151,7 +151,7 @@ typedef struct {
     size_t  workspace_bytes;     /* required size of the attention workspace              */
     int64_t mass_elems;          /* floats in block_mass: num_q_heads * sum_b nblk_b      */
     const int64_t* mass_off;     /* host [B+1], owned by the plan: sum of nblk over b' < b */
-    int32_t num_work_items;      /* CTAs of the segment-attention launch                  */
+    int32_t num_work_items;      /* work items of the segment kernels (their persistent CTAs claim them) */
     int32_t num_partial_rows;    /* (row, chunk) partial results merged at the end        */
     int64_t unique_kv_tokens;    /* valid tokens of the distinct segments referenced       */
     int64_t duplicated_kv_tokens;/* sum over branches of the tokens they attend to        */
