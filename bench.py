@@ -757,10 +757,12 @@ def decode_loop_measurement(rk, dev, workload: str, steps: int = 32):
     g = torch.Generator(device="cpu").manual_seed(77)
     k_new = torch.randn((B, lay0.num_kv_heads, d), generator=g).to(torch.bfloat16).to(dev)
     v_new = torch.randn((B, lay0.num_kv_heads, d), generator=g).to(torch.bfloat16).to(dev)
-    page_dev = torch.empty(B, dtype=torch.int32, device=dev)
-    slot_dev = torch.empty(B, dtype=torch.int32, device=dev)
-    page_host = torch.empty(B, dtype=torch.int32).pin_memory()
-    slot_host = torch.empty(B, dtype=torch.int32).pin_memory()
+    # (page, slot) of every step: a pinned row per step (the host runs ahead of the GPU, so a row that was
+    # reused would be overwritten before its copy has run) and one copy per step to the device
+    Bp = (B + 3) // 4 * 4                                      # rows 16-byte aligned
+    where_host = torch.empty((steps + 3, 2, Bp), dtype=torch.int32).pin_memory()
+    where_np = where_host.numpy()
+    where_dev = torch.empty((2, Bp), dtype=torch.int32, device=dev)
     new_pages = np.arange(nblk, nblk + B, dtype=np.int32)      # one spare page per branch per 16 steps
     plan = rk.rksc_plan_create(lay, t)
     out = torch.empty((B, Hq, d), dtype=torch.float32, device=dev)
@@ -770,11 +772,10 @@ def decode_loop_measurement(rk, dev, workload: str, steps: int = 32):
 
     def one(step, t):
         t, page, slot = rk.rksc_tables_append_token(t, new_pages + B * (step // 16))
-        page_host.copy_(torch.from_numpy(page))
-        slot_host.copy_(torch.from_numpy(slot))
-        page_dev.copy_(page_host, non_blocking=True)
-        slot_dev.copy_(slot_host, non_blocking=True)
-        rk.rksc_kv_append(lay, k_pool, v_pool, k_new, v_new, page_dev, slot_dev)
+        where_np[step, 0, :B] = page
+        where_np[step, 1, :B] = slot
+        where_dev.copy_(where_host[step], non_blocking=True)
+        rk.rksc_kv_append(lay, k_pool, v_pool, k_new, v_new, where_dev[0], where_dev[1])
         plan = rk.rksc_plan_create(lay, t)
         assert plan.workspace_bytes <= ws.numel() and plan.mass_elems <= mass.numel()
         rk.rksc_branch_decode_attention(plan, b.q, k_pool, v_pool, out=out, block_mass=mass, workspace=ws,
