@@ -93,11 +93,22 @@ cudaStream_t g_upload_stream[kMaxDevices];      // non-blocking: uploads do not 
 int32_t acquire_arena(int dev, size_t bytes, PlanArena* out) {
     {
         std::lock_guard<std::mutex> lock(g_mu);
+        // the smallest arena that fits and whose last plan has left the GPU: taking one that is still in
+        // use would make the caller wait for that plan's kernels (a decode loop that builds step i + 1's
+        // plan while step i runs would fall back into step with the GPU); rather a new arena then
         int best = -1;
-        for (int i = 0; i < (int)g_arena_pool.size(); ++i)
-            if (g_arena_pool[i].device == dev && g_arena_pool[i].capacity >= bytes &&
-                (best < 0 || g_arena_pool[i].capacity < g_arena_pool[best].capacity))
-                best = i;
+        for (int i = 0; i < (int)g_arena_pool.size(); ++i) {
+            PlanArena& c = g_arena_pool[i];
+            if (c.device != dev || c.capacity < bytes) continue;
+            if (c.busy) {
+                if (cudaEventQuery(c.done) != cudaSuccess) {
+                    cudaGetLastError();   // cudaErrorNotReady
+                    continue;
+                }
+                c.busy = false;
+            }
+            if (best < 0 || c.capacity < g_arena_pool[best].capacity) best = i;
+        }
         if (best >= 0) {
             *out = g_arena_pool[best];
             g_arena_pool.erase(g_arena_pool.begin() + best);
